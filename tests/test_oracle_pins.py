@@ -1,0 +1,361 @@
+"""Pins for the CPU oracle: it is checked against things other than itself.
+
+Hand-worked tie vectors, exact arithmetic done another way (float64 with a
+single rounding back to float32, Python integers, numpy int64 matmul, torch's
+bf16 cast), closed forms, invariants and brute force on tiny shapes. A dropped
+term, a wrong sign or index, a transposed operand, a reciprocal instead of a
+division, an FMA or a different association each fail at least one test here.
+"""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2606_14598_b200 import inputs as synth
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def f32(x):
+    return np.float32(x)
+
+
+def bf16_bits_of(x_f32: np.ndarray) -> np.ndarray:
+    """fp32 -> bf16 bit patterns through torch's cast (library routine, RNE)."""
+    t = torch.from_numpy(np.ascontiguousarray(x_f32, dtype=np.float32)).to(torch.bfloat16)
+    return synth.bf16_bits(t).copy()
+
+
+def bits_to_f64(bits: np.ndarray) -> np.ndarray:
+    return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def ordered(bits: np.ndarray) -> np.ndarray:
+    """Map bf16 bit patterns to integers that order like the values (+0 == -0)."""
+    b = bits.astype(np.int32)
+    return np.where(b & 0x8000, -(b & 0x7FFF), b)
+
+
+# --------------------------------------------------------------------------- quantizer
+
+def test_quantizer_hand_tie_vectors():
+    # absmax = 127 => s = 1 exactly, so q = rne(x): halves go to the even neighbour.
+    x = np.array([[127, 0.5, 1.5, 2.5, -0.5, -1.5, -2.5, 63.5, 126.5, -126.5, 0.375, 0.625, -127, 3.0]], np.float32)
+    want = np.array([[127, 0, 2, 2, 0, -2, -2, 64, 126, -126, 0, 1, -127, 3]], np.int8)
+    q, s = oracle.quantize_weight_per_channel(x)
+    assert s[0] == 1.0
+    assert (q == want).all()
+    # the same through the bf16 entry point (all values exact in bf16)
+    bits = bf16_bits_of(x)
+    assert (bits_to_f64(bits) == x.astype(np.float64)).all()
+    q2, s2 = oracle.quantize_act_per_token(bits)
+    assert s2[0] == 1.0 and (q2 == want).all()
+
+
+def test_quantizer_zero_row_and_mixed():
+    x = np.zeros((3, 16), np.float32)
+    x[1, 5] = -2.0
+    q, s = oracle.quantize_weight_per_channel(x)
+    assert s[0] == 1.0 and s[2] == 1.0 and (q[0] == 0).all() and (q[2] == 0).all()
+    assert s[1] == f32(2.0) / f32(127.0) and q[1, 5] == -127 and np.count_nonzero(q[1]) == 1
+
+
+def test_quantizer_division_not_reciprocal():
+    """s is amax/127 rounded once, and q uses x/s, each done another way here:
+    float64 division of two float32 values rounded back to float32 is the
+    correctly rounded float32 quotient (53 >= 2*24+2), and Python's round() is
+    round-half-to-even on the exact value."""
+    rng = np.random.default_rng(11)
+    x = rng.standard_normal((64, 257)).astype(np.float32)
+    x[:, 3] *= 20
+    q, s = oracle.quantize_weight_per_channel(x)
+    amax = np.abs(x).max(axis=1)
+    s_want = (amax.astype(np.float64) / 127.0).astype(np.float32)
+    assert (s == s_want).all()
+    r = (x.astype(np.float64) / s_want.astype(np.float64)[:, None]).astype(np.float32)
+    q_want = np.array([[max(-127, min(127, round(float(v)))) for v in row] for row in r], np.int64)
+    assert (q.astype(np.int64) == q_want).all()
+    # the reciprocal formulations are really different on this data (so the test can tell)
+    s_rcp = amax * f32(1.0 / 127.0)
+    q_rcp = np.rint(x * (f32(127.0) / amax)[:, None])
+    assert (s_rcp != s_want).any() or (q_rcp != q_want).any()
+
+
+def test_quantizer_bf16_matches_exact_route():
+    rng = np.random.default_rng(5)
+    a = rng.standard_normal((32, 384)).astype(np.float32)
+    a[:, 7] *= 20
+    bits = bf16_bits_of(a)
+    x = bits_to_f64(bits)                                   # exact values of the bf16 inputs
+    q, s = oracle.quantize_act_per_token(bits)
+    s_want = (np.abs(x).max(axis=1) / 127.0).astype(np.float32)
+    assert (s == s_want).all()
+    r = (x / s_want.astype(np.float64)[:, None]).astype(np.float32)
+    q_want = np.array([[round(float(v)) for v in row] for row in r], np.int64)
+    assert (q.astype(np.int64) == q_want).all()
+
+
+def test_quantizer_invariants():
+    rng = np.random.default_rng(3)
+    x = rng.standard_normal((128, 512)).astype(np.float32)
+    x[:, ::97] *= 20
+    q, s = oracle.quantize_weight_per_channel(x)
+    # every non-zero row uses the full range, and never -128
+    assert (np.abs(q.astype(np.int32)).max(axis=1) == 127).all()
+    assert q.min() >= -127
+    # the position of the absmax carries +-127 with the sign of x
+    j = np.abs(x).argmax(axis=1)
+    assert (q[np.arange(128), j] == 127 * np.sign(x[np.arange(128), j])).all()
+    # odd symmetry
+    qn, sn = oracle.quantize_weight_per_channel(-x)
+    assert (qn == -q).all() and (sn == s).all()
+    # power-of-two scaling commutes with every IEEE step
+    for j2 in (-7, 3, 20):
+        qs, ss = oracle.quantize_weight_per_channel(np.ldexp(x, j2).astype(np.float32))
+        assert (qs == q).all() and (ss == np.ldexp(s, j2)).all()
+    # permutation equivariance along K and along rows
+    pk = rng.permutation(512)
+    pr = rng.permutation(128)
+    qp, sp = oracle.quantize_weight_per_channel(np.ascontiguousarray(x[pr][:, pk]))
+    assert (qp == q[pr][:, pk]).all() and (sp == s[pr]).all()
+    # reconstruction error is at most half a step per element
+    err = np.abs(q.astype(np.float64) * s.astype(np.float64)[:, None] - x.astype(np.float64))
+    assert (err <= 0.5 * s.astype(np.float64)[:, None] * (1 + 1e-6)).all()
+
+
+def test_quantizer_leading_dimension_is_honoured():
+    # the ctypes wrapper passes dense arrays; check rows do not bleed into each other
+    x = np.zeros((2, 8), np.float32)
+    x[0] = [1, 2, 3, 4, 5, 6, 7, 8]
+    x[1] = [-80, 0, 0, 0, 0, 0, 0, 40]
+    q, s = oracle.quantize_weight_per_channel(x)
+    assert s[0] == f32(8) / f32(127) and s[1] == f32(80) / f32(127)
+    assert q[0, 7] == 127 and q[1, 0] == -127 and q[1, 7] in (63, 64)
+
+
+# --------------------------------------------------------------------------- integer GEMM
+
+def brute_gemm(qa, qw):
+    M, K = qa.shape
+    N = qw.shape[0]
+    acc = [[0] * N for _ in range(M)]
+    for k in range(K):                      # k outermost: a different loop order from the oracle
+        for n in range(N):
+            b = int(qw[n, k])
+            for m in range(M):
+                acc[m][n] += int(qa[m, k]) * b
+    return np.array(acc, dtype=np.int64).reshape(M, N)
+
+
+def test_gemm_brute_force_all_tiny_shapes():
+    rng = np.random.default_rng(0)
+    for M, N, K in itertools.product(range(1, 9), repeat=3):
+        qa = rng.integers(-127, 128, (M, K), dtype=np.int8)
+        qw = rng.integers(-127, 128, (N, K), dtype=np.int8)
+        assert (oracle.gemm_i32(qa, qw).astype(np.int64) == brute_gemm(qa, qw)).all(), (M, N, K)
+
+
+def test_gemm_not_transposed_on_nonsquare():
+    # A is [M,K], W is [N,K]: out[m,n] pairs row m of A with row n of W.
+    qa = np.array([[1, 2, 3], [4, 5, 6]], np.int8)              # M=2, K=3
+    qw = np.array([[1, 0, 0], [0, 1, 0], [0, 0, 1], [1, 1, 1]], np.int8)   # N=4
+    want = np.array([[1, 2, 3, 6], [4, 5, 6, 15]], np.int32)
+    assert (oracle.gemm_i32(qa, qw) == want).all()
+
+
+def test_gemm_identity_and_one_hot_weights():
+    rng = np.random.default_rng(1)
+    A = rng.standard_normal((16, 32)).astype(np.float32)
+    qa, _ = oracle.quantize_act_per_token(bf16_bits_of(A))
+    c = 0.37
+    W = (c * np.eye(32)).astype(np.float32)
+    qw, s_ch = oracle.quantize_weight_per_channel(W)
+    assert (qw == 127 * np.eye(32, dtype=np.int8)).all()
+    assert (s_ch == f32(c) / f32(127)).all()
+    assert (oracle.gemm_i32(qa, qw) == 127 * qa.astype(np.int32)).all()
+    # one-hot rows pick (and scale) columns of qa
+    pick = rng.integers(0, 32, 10)
+    W1 = np.zeros((10, 32), np.float32)
+    W1[np.arange(10), pick] = -2.5
+    qw1, _ = oracle.quantize_weight_per_channel(W1)
+    assert (oracle.gemm_i32(qa, qw1) == -127 * qa[:, pick].astype(np.int32)).all()
+
+
+def test_gemm_library_matmul_medium():
+    rng = np.random.default_rng(2)
+    qa = rng.integers(-127, 128, (37, 1000), dtype=np.int8)
+    qw = rng.integers(-127, 128, (53, 1000), dtype=np.int8)
+    want = qa.astype(np.int64) @ qw.astype(np.int64).T
+    assert (oracle.gemm_i32(qa, qw).astype(np.int64) == want).all()
+    # K-split additivity
+    a1 = oracle.gemm_i32(np.ascontiguousarray(qa[:, :336]), np.ascontiguousarray(qw[:, :336]))
+    a2 = oracle.gemm_i32(np.ascontiguousarray(qa[:, 336:]), np.ascontiguousarray(qw[:, 336:]))
+    assert (a1.astype(np.int64) + a2 == want).all()
+
+
+def test_gemm_overflow_edge_closed_form():
+    # K * 127^2 < 2^31 holds up to K = 133144 and fails at 133145.
+    assert oracle.K_MAX * 127 * 127 < 2 ** 31 <= (oracle.K_MAX + 1) * 127 * 127
+    for K in (133136, oracle.K_MAX):
+        qa = np.full((2, K), 127, np.int8)
+        qa[1] = -127
+        qw = np.full((3, K), 127, np.int8)
+        qw[2] = -127
+        acc = oracle.gemm_i32(qa, qw)
+        v = K * 16129
+        assert acc.tolist() == [[v, v, -v], [-v, -v, v]]
+    K = oracle.K_MAX + 1
+    with pytest.raises(OverflowError):
+        oracle.gemm_i32(np.full((1, K), 127, np.int8), np.full((1, K), 127, np.int8))
+    # -128 codes stay exact through K = 131071 (K * 2^14 < 2^31)
+    K = 131071
+    acc = oracle.gemm_i32(np.full((1, K), -128, np.int8), np.full((1, K), -128, np.int8))
+    assert acc[0, 0] == K * 16384
+
+
+# --------------------------------------------------------------------------- epilogue
+
+def step_f32(acc, s_tok, s_ch, bias):
+    """The epilogue's fp32 value via float64 steps, each rounded once to float32.
+    A float64 product of two float32 values is exact, and a float64 sum of two
+    float32 values rounds innocuously, so each step is the IEEE float32 result."""
+    t = acc.astype(np.float32)                                           # int32 -> fp32 RNE (numpy cast)
+    t = (t.astype(np.float64) * s_tok.astype(np.float64)[:, None]).astype(np.float32)
+    t = (t.astype(np.float64) * s_ch.astype(np.float64)[None, :]).astype(np.float32)
+    if bias is not None:
+        t = (t.astype(np.float64) + bias.astype(np.float64)[None, :]).astype(np.float32)
+    return t
+
+
+def test_epilogue_hand_vectors():
+    one = np.ones((1,), np.float32)
+    zero = np.zeros((1,), np.float32)
+    # bf16 ties: 257 sits between 256 (even mantissa) and 258; 259 between 258 and 260 (even)
+    for a, want in ((257, 256.0), (259, 260.0), (258, 258.0), (-257, -256.0), (-259, -260.0), (0, 0.0)):
+        out = oracle.epilogue(np.array([[a]], np.int32), one, one, zero)
+        assert bits_to_f64(out)[0, 0] == want
+    # int32 -> fp32 rounds to nearest even above 2^24, then bf16 rounds again
+    out = oracle.epilogue(np.array([[2 ** 24 + 1, 2 ** 24 + 3, 2 ** 31 - 1, -2 ** 31]], np.int32), one,
+                          np.ones((4,), np.float32), None)
+    assert bits_to_f64(out)[0].tolist() == [2.0 ** 24, 2.0 ** 24, 2.0 ** 31, -2.0 ** 31]
+    # bias only
+    b = np.array([0.01171875, -3.0], np.float32)
+    out = oracle.epilogue(np.zeros((1, 2), np.int32), one, np.ones((2,), np.float32), b)
+    assert bits_to_f64(out)[0].tolist() == [0.01171875, -3.0]
+
+
+def test_epilogue_no_fma_and_left_to_right():
+    # (1 * (1+2^-12)) * (1+2^-12) = 1 + 2^-11 + 2^-24 exactly: the last term is half an ulp and
+    # the tie goes down to 1 + 2^-11. Adding bias = -(1 + 2^-11) gives 0 with a rounded product,
+    # 2^-24 if the multiply-add were fused.
+    e = f32(1.0) + f32(2.0 ** -12)
+    bias = np.array([-(1.0 + 2.0 ** -11)], np.float32)
+    out = oracle.epilogue(np.array([[1]], np.int32), np.array([e], np.float32), np.array([e], np.float32), bias)
+    assert bits_to_f64(out)[0, 0] == 0.0
+    # association: triples (found by search) where (a*s)*c and a*(s*c) land on different bf16
+    # values; the left-to-right result is required. Expected bits were worked out through
+    # float64 steps each rounded once to float32, and are re-derived below.
+    cases = [(-6918, "0x1.b99f02p-5", "0x1.09a68p-12", 0xBDC2, 0xBDC1),
+             (-47474, "0x1.cbeebap-5", "0x1.5c123ep-11", 0xBFE2, 0xBFE3),
+             (-16675, "0x1.5cc1a6p-6", "0x1.1fc4fcp-11", 0xBE48, 0xBE47),
+             (6760, "0x1.4b91dp-5", "0x1.4a47ep-11", 0x3E30, 0x3E31),
+             (89821, "0x1.7a5ac6p-5", "0x1.f69036p-12", 0x3FFF, 0x3FFE)]
+    for a, s_hex, c_hex, left_bits, right_bits in cases:
+        s_tok = np.array([float.fromhex(s_hex)], np.float32)
+        s_ch = np.array([float.fromhex(c_hex)], np.float32)
+        assert float(s_tok[0]) == float.fromhex(s_hex) and float(s_ch[0]) == float.fromhex(c_hex)
+        acc = np.array([[a]], np.int32)
+        left = bf16_bits_of(step_f32(acc, s_tok, s_ch, None))[0, 0]
+        sc = np.float32(np.float64(s_tok[0]) * np.float64(s_ch[0]))
+        right = bf16_bits_of(np.array([np.float32(np.float64(a) * np.float64(sc))]))[0]
+        assert (left, right) == (left_bits, right_bits)
+        assert oracle.epilogue(acc, s_tok, s_ch, None)[0, 0] == left_bits
+
+
+def test_epilogue_matches_stepwise_float64_route_and_bound():
+    rng = np.random.default_rng(4)
+    M, N = 64, 96
+    acc = rng.integers(-80000, 80000, (M, N)).astype(np.int32)
+    s_tok = (rng.random(M) * 0.3 + 0.02).astype(np.float32)
+    s_ch = (rng.random(N) * 0.0008 + 0.0002).astype(np.float32)
+    bias = (rng.standard_normal(N) * 0.01).astype(np.float32)
+    out = oracle.epilogue(acc, s_tok, s_ch, bias)
+    assert (out == bf16_bits_of(step_f32(acc, s_tok, s_ch, bias))).all()
+    # against the unrounded value: at most one bf16 step away, except under cancellation
+    exact = acc.astype(np.float64) * s_tok.astype(np.float64)[:, None] * s_ch.astype(np.float64)[None, :] + bias
+    near = bf16_bits_of(exact.astype(np.float32))
+    cancel = np.abs(exact) < 2.0 ** -6 * np.abs(bias)[None, :]
+    assert (np.abs(ordered(out) - ordered(near))[~cancel] <= 1).all()
+    rel = np.abs(bits_to_f64(out) - exact)[~cancel] / np.abs(exact)[~cancel]
+    assert rel.max() <= 2.0 ** -8 * (1 + 1e-3)
+    # no bias: NULL pointer path equals a zero bias... except for the sign of zero
+    out0 = oracle.epilogue(acc, s_tok, s_ch, None)
+    assert (out0 == bf16_bits_of(step_f32(acc, s_tok, s_ch, None))).all()
+
+
+# --------------------------------------------------------------------------- whole path
+
+def float_linear(A_bits, W, bias):
+    return bits_to_f64(A_bits) @ W.astype(np.float64).T + bias.astype(np.float64)[None, :]
+
+
+def test_fused_equals_its_steps_and_is_finite():
+    spec = synth.CONFIGS["c1"][0]
+    t = synth.make_linear(spec)
+    A_bits = synth.bf16_bits(t["A"])
+    qw, s_ch = oracle.quantize_weight_per_channel(t["W"].numpy())
+    r = oracle.linear_fused_bf16(A_bits, qw, s_ch, t["bias"].numpy())
+    qa, s_tok = oracle.quantize_act_per_token(A_bits)
+    assert (r["qa"] == qa).all() and (r["s_tok"] == s_tok).all()
+    acc = oracle.gemm_i32(qa, qw)
+    assert (r["acc"] == acc).all()
+    assert (r["out"] == oracle.epilogue(acc, s_tok, s_ch, t["bias"].numpy())).all()
+    r2 = oracle.linear_fused_int8(qa, s_tok, qw, s_ch, t["bias"].numpy())
+    assert (r2["out"] == r["out"]).all()
+    out = bits_to_f64(r["out"])
+    assert np.isfinite(out).all()
+    ref = float_linear(A_bits, t["W"].numpy(), t["bias"].numpy())
+    cos = (out * ref).sum() / math.sqrt((out * out).sum() * (ref * ref).sum())
+    assert cos > 0.9995
+
+
+def test_error_shrinks_as_outliers_vanish():
+    """Dequantized output approaches the float matmul as the outlier multiplier goes to 1, and at 1
+    the error matches the uniform-rounding closed form sqrt(e_a^2 + e_w^2), e = (E absmax / 127)/sqrt(12)."""
+    M, K, N = 96, 3072, 128
+    errs = []
+    for mult in (20.0, 10.0, 5.0, 2.0, 1.0):
+        spec = synth.LinearSpec("vanish", M, K, N, outlier_frac=0.01, outlier_mult=mult)
+        t = synth.make_linear(spec)
+        A_bits = synth.bf16_bits(t["A"])
+        W, b = t["W"].numpy(), t["bias"].numpy()
+        qw, s_ch = oracle.quantize_weight_per_channel(W)
+        out = bits_to_f64(oracle.linear_fused_bf16(A_bits, qw, s_ch, b)["out"])
+        ref = float_linear(A_bits, W, b)
+        errs.append(np.linalg.norm(out - ref) / np.linalg.norm(ref))
+    assert all(a > b for a, b in zip(errs, errs[1:])), errs
+    assert errs[0] > 0.03 and errs[-1] < 0.016, errs
+    # closed form at multiplier 1: E[absmax of 3072 N(0,1)] ~ 3.6 => e ~ 3.6/127/sqrt(12) = 0.0082 each
+    e = 3.6 / 127 / math.sqrt(12)
+    assert abs(errs[-1] - math.sqrt(2) * e) < 0.2 * math.sqrt(2) * e, errs
+
+
+def test_generator_is_seeded_and_shaped():
+    spec = synth.CONFIGS["c2"][0]
+    ch = synth.outlier_channels(spec)
+    assert ch.size == 31 or ch.size == 30
+    small = synth.LinearSpec(spec.name, 64, spec.K, 8)
+    a1 = synth.make_activations(small)
+    a2 = synth.make_activations(small)
+    assert torch.equal(a1, a2)
+    assert not torch.equal(a1, synth.make_activations(small, seed=1))
+    std = a1.float().std(dim=0)
+    mask = np.zeros(spec.K, bool)
+    mask[synth.outlier_channels(small)] = True
+    assert std[torch.from_numpy(mask)].mean() > 15 and std[torch.from_numpy(~mask)].mean() < 1.3
+    g = synth.make_activations(synth.LinearSpec("g", 64, 1024, 8, act="gelu", outlier_frac=0.0))
+    assert g.float().min() > -0.18 and g.float().max() > 2.0
