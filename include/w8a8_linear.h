@@ -1,0 +1,165 @@
+/*
+ * w8a8_linear.h -- C ABI of the B200 (sm_100a) fused W8A8 linear layer.
+ *
+ * The layer follows the paper's Method section: "The quantization recipe
+ * (reused)" (per-channel symmetric int8 weights, per-token dynamic int8
+ * activations) and "The fused kernel" (int8 x int8 -> int32 accumulation on
+ * the tensor cores; per-token scale, per-channel scale and bias applied off the
+ * int32 accumulator in the GEMM epilogue; one pass, dequantized output).
+ *
+ * Arithmetic, fixed for every entry point (IEEE binary32, round to nearest
+ * even, no fused multiply-add, no flush to zero):
+ *     s      = amax > 0 ? amax / 127 : 1           one division per row
+ *     q[k]   = clamp(rne(x[k] / s), -127, 127)     one division per element
+ *     acc    = sum_k qa[m,k] * qw[n,k]             exact, int32
+ *     out    = bf16(((float(acc) * s_tok[m]) * s_ch[n]) + bias[n])
+ * Inputs must be finite; NaN/Inf give unspecified values (never a hang or an
+ * out-of-bounds access).
+ *
+ * Conventions for all calls:
+ *   - Matrices are row-major. A is [M,K], W and qw are [N,K], out is [M,N];
+ *     ld* are row strides in ELEMENTS.
+ *   - Unless a parameter says "host", every pointer is a DEVICE pointer that the
+ *     caller owns (allocated by the caller, e.g. through PyTorch). The library
+ *     allocates no device memory and keeps no reference after the call's work
+ *     has run.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Calls only enqueue work on it and return; they do not synchronize unless
+ *     stated.
+ *   - The return value is a w8a8_status. Argument errors are detected before
+ *     anything is enqueued. There is no CPU fallback and no other backend: on a
+ *     device that is not sm_100 the compute calls return W8A8_ERR_ARCH.
+ */
+#ifndef W8A8_LINEAR_H_
+#define W8A8_LINEAR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum w8a8_status {
+    W8A8_OK = 0,
+    W8A8_ERR_INVALID_ARG = 1, /* NULL pointer, M/N/K <= 0, ld smaller than the row, unknown dtype */
+    W8A8_ERR_ALIGNMENT = 2,   /* pointer not 16-byte aligned, or K/N/ld break the 16-byte rules below */
+    W8A8_ERR_K_OVERFLOW = 3,  /* K > 133144: K * 127^2 would not fit in int32 */
+    W8A8_ERR_WORKSPACE = 4,   /* workspace NULL or smaller than int8_linear_workspace_bytes() */
+    W8A8_ERR_ARCH = 5,        /* current device is not compute capability 10.x */
+    W8A8_ERR_CUDA = 6,        /* a CUDA runtime/driver call failed (launch, descriptor encode) */
+    W8A8_ERR_TIMEOUT = 7      /* a bounded device-side wait expired (reported by int8_check_status) */
+} w8a8_status;
+
+/* activation dtype selector of int8_linear_fused */
+enum { W8A8_ACT_BF16 = 0, W8A8_ACT_INT8 = 1 };
+
+/* Largest K the integer path accepts (K * 127^2 < 2^31). */
+#define W8A8_K_MAX 133144
+
+/*
+ * Per-output-channel weight quantization (Method, "The quantization recipe":
+ * per-channel int8 weights). Offline set-up step.
+ *   W     in   fp32 [N,K], row stride ldw (elements, >= K, multiple of 4), 16-byte aligned
+ *   qw    out  int8 [N,K] dense (row stride K), 16-byte aligned
+ *   s_ch  out  fp32 [N]
+ * Requires K % 16 == 0.
+ */
+int int8_quantize_weight_per_channel(const float* W, int64_t N, int64_t K, int64_t ldw,
+                                     int8_t* qw, float* s_ch, void* stream);
+
+/*
+ * Per-token activation quantization (Method, "The fused kernel": per-token
+ * scales are dynamic, computed online from the activations).
+ *   A_bf16 in   bf16 [M,K], row stride lda (elements, >= K, multiple of 8), 16-byte aligned
+ *   qa     out  int8 [M,K] dense, 16-byte aligned
+ *   s_tok  out  fp32 [M]
+ * Requires K % 16 == 0.
+ */
+int int8_quantize_act_per_token(const void* A_bf16, int64_t M, int64_t K, int64_t lda,
+                                int8_t* qa, float* s_tok, void* stream);
+
+/*
+ * Bytes of caller-provided device workspace int8_linear_fused needs for this
+ * problem (0 on invalid sizes). Layout, from the workspace base (which must be
+ * 256-byte aligned): a 256-byte status block; then, for bf16 activations only,
+ * s_tok as fp32 [M] (padded to 256 bytes) and qa as int8 [M,K] dense. After a
+ * bf16 call the caller may read qa and s_tok back from there
+ * (int8_linear_workspace_offsets gives the byte offsets).
+ */
+size_t int8_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int a_dtype);
+
+/* Byte offsets of s_tok and qa inside the workspace for bf16 activations. */
+void int8_linear_workspace_offsets(int64_t M, int64_t K, size_t* s_tok_offset, size_t* qa_offset);
+
+/*
+ * The fused W8A8 linear (Method, "The fused kernel"):
+ *     out[m,n] = bf16(acc[m,n] * s_tok[m] * s_ch[n] + bias[n]),
+ *     acc = qa . qw^T in int32 on the tensor cores.
+ *   A         in   a_dtype == W8A8_ACT_BF16: bf16 [M,K], quantized per token inside the call;
+ *                  a_dtype == W8A8_ACT_INT8: int8 [M,K] codes in [-127,127] (-128 is tolerated
+ *                  and exact while K <= 131071). Row stride lda elements; 16-byte aligned;
+ *                  lda bytes a multiple of 16.
+ *   s_tok_in  in   fp32 [M]; required iff a_dtype == W8A8_ACT_INT8, else must be NULL
+ *   qw        in   int8 [N,K] dense, 16-byte aligned
+ *   s_ch      in   fp32 [N]
+ *   bias      in   fp32 [N] or NULL (no bias term)
+ *   out_bf16  out  bf16 [M,N], row stride ldo elements (multiple of 8), 16-byte aligned
+ *   workspace      device scratch of at least int8_linear_workspace_bytes(); two calls that
+ *                  may overlap on the device need distinct workspaces
+ * Requires K % 16 == 0, N % 8 == 0, K <= W8A8_K_MAX. The kernel configuration
+ * (tile shape, pipeline depth, skinny-M path) is chosen from (M,N,K); the
+ * paper's per-shape autotuning ("Why autotuning is load-bearing") is replaced
+ * by a static per-shape table.
+ */
+int int8_linear_fused(const void* A, int a_dtype, int64_t lda, const float* s_tok_in,
+                      const int8_t* qw, const float* s_ch, const float* bias,
+                      void* out_bf16, int64_t ldo, int64_t M, int64_t N, int64_t K,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Same computation with the activations and the result in HOST memory
+ * (pinned memory makes the copies asynchronous): copies A to d_A, runs
+ * int8_linear_fused on bf16 activations, copies the result to out_host, all on
+ * `stream`, and returns without synchronizing.
+ *   A_host   in   host bf16 [M,K] dense        d_A    device bf16 [M,K] staging (caller-owned)
+ *   out_host out  host bf16 [M,N] dense        d_out  device bf16 [M,N] staging (caller-owned)
+ * Weights, scales, bias and workspace are device pointers as above.
+ */
+int int8_linear_fused_host(const void* A_host, void* d_A,
+                           const int8_t* qw, const float* s_ch, const float* bias,
+                           void* d_out, void* out_host, int64_t M, int64_t N, int64_t K,
+                           void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Test-only export of the raw accumulators of the tensor-core path (the int32
+ * values the fused epilogue consumes): acc[m,n] = sum_k qa[m,k] * qw[n,k].
+ *   qa in int8 [M,K] dense; qw in int8 [N,K] dense; acc out int32 [M,N] dense (N % 4 == 0);
+ *   workspace as for int8_linear_fused with W8A8_ACT_INT8.
+ */
+int int8_gemm_i32_debug(const int8_t* qa, const int8_t* qw, int32_t* acc,
+                        int64_t M, int64_t N, int64_t K,
+                        void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Synchronizes `stream` and returns the device-side status word of `workspace`:
+ * W8A8_OK, or W8A8_ERR_TIMEOUT if a bounded wait inside a kernel gave up (the
+ * kernel then released its resources and returned; outputs are undefined).
+ * Clears the word. Returns W8A8_ERR_CUDA if the synchronize failed.
+ */
+int int8_check_status(void* workspace, void* stream);
+
+/* Force a kernel configuration for sweeps (-1 = choose from the shape). Returns the previous value. */
+int int8_linear_force_config(int config_id);
+
+/* Number of kernel configurations, and a short description of one (NULL if out of range). */
+int int8_linear_num_configs(void);
+const char* int8_linear_config_name(int config_id);
+
+/* Static string for a status code. */
+const char* int8_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* W8A8_LINEAR_H_ */

@@ -1,0 +1,203 @@
+// C ABI of the library: argument validation, workspace layout, dispatch.
+// No device memory is allocated here and nothing falls back to the CPU.
+#include "../../include/w8a8_linear.h"
+#include "internal.h"
+
+#include <atomic>
+#include <cstdint>
+
+namespace {
+
+using namespace w8a8;
+
+constexpr size_t kStatusBlock = 256;
+constexpr int kSkinnyM = 16;          // at or below this many tokens the weight-streaming path runs
+
+std::atomic<int> g_forced_config{-1};
+
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_arch() {
+    static thread_local int cached_dev = -1;
+    static thread_local int cached_ok = 0;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return W8A8_ERR_CUDA;
+    if (dev != cached_dev) {
+        int major = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return W8A8_ERR_CUDA;
+        cached_dev = dev;
+        cached_ok = (major == 10);
+    }
+    return cached_ok ? W8A8_OK : W8A8_ERR_ARCH;
+}
+
+int check_dims(int64_t M, int64_t N, int64_t K) {
+    if (M <= 0 || N <= 0 || K <= 0) return W8A8_ERR_INVALID_ARG;
+    if (M > INT32_MAX || N > INT32_MAX) return W8A8_ERR_INVALID_ARG;
+    if (K > W8A8_K_MAX) return W8A8_ERR_K_OVERFLOW;
+    if (K % 16 != 0) return W8A8_ERR_ALIGNMENT;
+    return W8A8_OK;
+}
+
+void offsets(int64_t M, size_t* s_tok_off, size_t* qa_off) {
+    *s_tok_off = kStatusBlock;
+    *qa_off = kStatusBlock + round_up(static_cast<size_t>(M) * sizeof(float), 256);
+}
+
+} // namespace
+
+extern "C" {
+
+const char* int8_status_string(int status) {
+    switch (status) {
+        case W8A8_OK: return "ok";
+        case W8A8_ERR_INVALID_ARG: return "invalid argument";
+        case W8A8_ERR_ALIGNMENT: return "alignment: pointers must be 16-byte aligned, K % 16 == 0, N % 8 == 0, row strides multiples of 16 bytes";
+        case W8A8_ERR_K_OVERFLOW: return "K too large: K * 127^2 must stay below 2^31";
+        case W8A8_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case W8A8_ERR_ARCH: return "device is not sm_100 (B200)";
+        case W8A8_ERR_CUDA: return "CUDA call failed";
+        case W8A8_ERR_TIMEOUT: return "a bounded device-side wait expired";
+        default: return "unknown status";
+    }
+}
+
+int int8_linear_force_config(int config_id) { return g_forced_config.exchange(config_id); }
+int int8_linear_num_configs(void) { return tc_num_configs() + 1; }
+const char* int8_linear_config_name(int config_id) {
+    if (config_id == tc_num_configs()) return "simt dp4a (skinny M / cross-check)";
+    return tc_config_name(config_id);
+}
+
+int int8_quantize_weight_per_channel(const float* W, int64_t N, int64_t K, int64_t ldw,
+                                     int8_t* qw, float* s_ch, void* stream) {
+    if (W == nullptr || qw == nullptr || s_ch == nullptr) return W8A8_ERR_INVALID_ARG;
+    if (N <= 0 || K <= 0 || N > INT32_MAX || K > INT32_MAX || ldw < K) return W8A8_ERR_INVALID_ARG;
+    if (K % 16 != 0 || ldw % 4 != 0 || !aligned16(W) || !aligned16(qw)) return W8A8_ERR_ALIGNMENT;
+    if (int e = check_arch()) return e;
+    cudaError_t ce = launch_quantize_f32(W, ldw, static_cast<int>(N), static_cast<int>(K), qw, s_ch,
+                                         static_cast<cudaStream_t>(stream));
+    return ce == cudaSuccess ? W8A8_OK : W8A8_ERR_CUDA;
+}
+
+int int8_quantize_act_per_token(const void* A_bf16, int64_t M, int64_t K, int64_t lda,
+                                int8_t* qa, float* s_tok, void* stream) {
+    if (A_bf16 == nullptr || qa == nullptr || s_tok == nullptr) return W8A8_ERR_INVALID_ARG;
+    if (M <= 0 || K <= 0 || M > INT32_MAX || K > INT32_MAX || lda < K) return W8A8_ERR_INVALID_ARG;
+    if (K % 16 != 0 || lda % 8 != 0 || !aligned16(A_bf16) || !aligned16(qa)) return W8A8_ERR_ALIGNMENT;
+    if (int e = check_arch()) return e;
+    cudaError_t ce = launch_quantize_bf16(A_bf16, lda, static_cast<int>(M), static_cast<int>(K), qa, s_tok, nullptr,
+                                          static_cast<cudaStream_t>(stream));
+    return ce == cudaSuccess ? W8A8_OK : W8A8_ERR_CUDA;
+}
+
+size_t int8_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int a_dtype) {
+    if (M <= 0 || N <= 0 || K <= 0) return 0;
+    if (a_dtype == W8A8_ACT_INT8) return kStatusBlock;
+    if (a_dtype != W8A8_ACT_BF16) return 0;
+    size_t s_off, q_off;
+    offsets(M, &s_off, &q_off);
+    return q_off + round_up(static_cast<size_t>(M) * static_cast<size_t>(K), 256);
+}
+
+void int8_linear_workspace_offsets(int64_t M, int64_t K, size_t* s_tok_offset, size_t* qa_offset) {
+    (void)K;
+    size_t s_off, q_off;
+    offsets(M, &s_off, &q_off);
+    if (s_tok_offset) *s_tok_offset = s_off;
+    if (qa_offset) *qa_offset = q_off;
+}
+
+int int8_linear_fused(const void* A, int a_dtype, int64_t lda, const float* s_tok_in,
+                      const int8_t* qw, const float* s_ch, const float* bias,
+                      void* out_bf16, int64_t ldo, int64_t M, int64_t N, int64_t K,
+                      void* workspace, size_t workspace_bytes, void* stream) {
+    if (A == nullptr || qw == nullptr || s_ch == nullptr || out_bf16 == nullptr) return W8A8_ERR_INVALID_ARG;
+    if (a_dtype != W8A8_ACT_BF16 && a_dtype != W8A8_ACT_INT8) return W8A8_ERR_INVALID_ARG;
+    if ((a_dtype == W8A8_ACT_INT8) != (s_tok_in != nullptr)) return W8A8_ERR_INVALID_ARG;
+    if (int e = check_dims(M, N, K)) return e;
+    if (lda < K || ldo < N) return W8A8_ERR_INVALID_ARG;
+    const int64_t lda_bytes = lda * (a_dtype == W8A8_ACT_BF16 ? 2 : 1);
+    if (N % 8 != 0 || ldo % 8 != 0 || lda_bytes % 16 != 0) return W8A8_ERR_ALIGNMENT;
+    if (!aligned16(A) || !aligned16(qw) || !aligned16(out_bf16)) return W8A8_ERR_ALIGNMENT;
+    if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0 ||
+        workspace_bytes < int8_linear_workspace_bytes(M, N, K, a_dtype))
+        return W8A8_ERR_WORKSPACE;
+    if (int e = check_arch()) return e;
+
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    int* status = reinterpret_cast<int*>(ws);
+
+    GemmArgs g{};
+    g.qw = qw; g.s_ch = s_ch; g.bias = bias; g.out = out_bf16; g.ldo = ldo;
+    g.M = static_cast<int>(M); g.N = static_cast<int>(N); g.K = static_cast<int>(K);
+    g.raw_i32 = false; g.status = status;
+    if (a_dtype == W8A8_ACT_BF16) {
+        size_t s_off, q_off;
+        offsets(M, &s_off, &q_off);
+        float* s_tok = reinterpret_cast<float*>(ws + s_off);
+        int8_t* qa = reinterpret_cast<int8_t*>(ws + q_off);
+        if (launch_quantize_bf16(A, lda, g.M, g.K, qa, s_tok, status, st) != cudaSuccess) return W8A8_ERR_CUDA;
+        g.qa = qa; g.lda_q = K; g.s_tok = s_tok; g.after_quantizer = true;
+    } else {
+        if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return W8A8_ERR_CUDA;
+        g.qa = static_cast<const int8_t*>(A); g.lda_q = lda; g.s_tok = s_tok_in; g.after_quantizer = false;
+    }
+    const int forced = g_forced_config.load();
+    if ((forced < 0 && M <= kSkinnyM) || forced == tc_num_configs())
+        return launch_gemm_simt(g, st) == cudaSuccess ? W8A8_OK : W8A8_ERR_CUDA;
+    return launch_gemm_tc(g, forced, st);
+}
+
+int int8_linear_fused_host(const void* A_host, void* d_A,
+                           const int8_t* qw, const float* s_ch, const float* bias,
+                           void* d_out, void* out_host, int64_t M, int64_t N, int64_t K,
+                           void* workspace, size_t workspace_bytes, void* stream) {
+    if (A_host == nullptr || d_A == nullptr || d_out == nullptr || out_host == nullptr) return W8A8_ERR_INVALID_ARG;
+    if (int e = check_dims(M, N, K)) return e;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(d_A, A_host, static_cast<size_t>(M) * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return W8A8_ERR_CUDA;
+    int e = int8_linear_fused(d_A, W8A8_ACT_BF16, K, nullptr, qw, s_ch, bias, d_out, N, M, N, K,
+                              workspace, workspace_bytes, stream);
+    if (e != W8A8_OK) return e;
+    if (cudaMemcpyAsync(out_host, d_out, static_cast<size_t>(M) * N * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return W8A8_ERR_CUDA;
+    return W8A8_OK;
+}
+
+int int8_gemm_i32_debug(const int8_t* qa, const int8_t* qw, int32_t* acc,
+                        int64_t M, int64_t N, int64_t K,
+                        void* workspace, size_t workspace_bytes, void* stream) {
+    if (qa == nullptr || qw == nullptr || acc == nullptr) return W8A8_ERR_INVALID_ARG;
+    if (int e = check_dims(M, N, K)) return e;
+    if (N % 4 != 0 || !aligned16(qa) || !aligned16(qw) || !aligned16(acc)) return W8A8_ERR_ALIGNMENT;
+    if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0 || workspace_bytes < kStatusBlock)
+        return W8A8_ERR_WORKSPACE;
+    if (int e = check_arch()) return e;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int* status = static_cast<int*>(workspace);
+    if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return W8A8_ERR_CUDA;
+    GemmArgs g{};
+    g.qa = qa; g.lda_q = K; g.s_tok = nullptr; g.qw = qw; g.s_ch = nullptr; g.bias = nullptr;
+    g.out = acc; g.ldo = N; g.M = static_cast<int>(M); g.N = static_cast<int>(N); g.K = static_cast<int>(K);
+    g.raw_i32 = true; g.status = status; g.after_quantizer = false;
+    const int forced = g_forced_config.load();
+    if ((forced < 0 && M <= kSkinnyM) || forced == tc_num_configs())
+        return launch_gemm_simt(g, st) == cudaSuccess ? W8A8_OK : W8A8_ERR_CUDA;
+    return launch_gemm_tc(g, forced, st);
+}
+
+int int8_check_status(void* workspace, void* stream) {
+    if (workspace == nullptr) return W8A8_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int word = 0;
+    if (cudaMemcpyAsync(&word, workspace, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return W8A8_ERR_CUDA;
+    if (cudaMemsetAsync(workspace, 0, sizeof(int), st) != cudaSuccess) return W8A8_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return W8A8_ERR_CUDA;
+    return word & 0xff;
+}
+
+} // extern "C"

@@ -1,0 +1,116 @@
+// CUDA-core (dp4a) W8A8 GEMM + epilogue. Two uses:
+//   * skinny M (a handful of tokens, e.g. the adaLN modulation linear): the
+//     work is streaming the int8 weights once from HBM, which this does with
+//     128-bit loads, several rows in flight per warp;
+//   * an exact second implementation of acc / out for any shape (slow), used
+//     to cross-check the tensor-core path on the device.
+// Each warp owns NPW consecutive output channels and MB rows of A; lanes split K.
+#include "internal.h"
+#include "ptx.cuh"
+
+#include <cuda_bf16.h>
+
+namespace w8a8 {
+namespace {
+
+__device__ __forceinline__ int dot16(const uint4& a, const uint4& b, int acc) {
+    acc = __dp4a(static_cast<int>(a.x), static_cast<int>(b.x), acc);
+    acc = __dp4a(static_cast<int>(a.y), static_cast<int>(b.y), acc);
+    acc = __dp4a(static_cast<int>(a.z), static_cast<int>(b.z), acc);
+    acc = __dp4a(static_cast<int>(a.w), static_cast<int>(b.w), acc);
+    return acc;
+}
+
+template <int MB, int NPW, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32)
+gemm_simt_kernel(const int8_t* __restrict__ qa, int64_t lda_q, const float* __restrict__ s_tok,
+                 const int8_t* __restrict__ qw, const float* __restrict__ s_ch, const float* __restrict__ bias,
+                 void* __restrict__ out, int64_t ldo, int M, int N, int K, int raw_i32, int after_quantizer) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n0 = (blockIdx.x * WARPS + warp) * NPW;
+    const int m0 = blockIdx.y * MB;
+    if (n0 >= N) return;
+
+    int acc[MB][NPW];
+#pragma unroll
+    for (int i = 0; i < MB; ++i)
+#pragma unroll
+        for (int j = 0; j < NPW; ++j) acc[i][j] = 0;
+
+    const int8_t* wrow[NPW];
+#pragma unroll
+    for (int j = 0; j < NPW; ++j) wrow[j] = qw + static_cast<int64_t>(min(n0 + j, N - 1)) * K;
+    const int8_t* arow[MB];
+#pragma unroll
+    for (int i = 0; i < MB; ++i) arow[i] = qa + static_cast<int64_t>(min(m0 + i, M - 1)) * lda_q;
+
+    // weights do not depend on the quantizer: warm the first chunk before waiting for it
+    if (after_quantizer) grid_dep_wait();
+
+    for (int k = lane * 16; k < K; k += 32 * 16) {
+        uint4 w[NPW], a[MB];
+#pragma unroll
+        for (int j = 0; j < NPW; ++j) w[j] = __ldg(reinterpret_cast<const uint4*>(wrow[j] + k));
+#pragma unroll
+        for (int i = 0; i < MB; ++i) a[i] = *reinterpret_cast<const uint4*>(arow[i] + k);
+#pragma unroll
+        for (int i = 0; i < MB; ++i)
+#pragma unroll
+            for (int j = 0; j < NPW; ++j) acc[i][j] = dot16(a[i], w[j], acc[i][j]);
+    }
+#pragma unroll
+    for (int i = 0; i < MB; ++i)
+#pragma unroll
+        for (int j = 0; j < NPW; ++j)
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) acc[i][j] += __shfl_xor_sync(0xffffffffu, acc[i][j], o);
+
+    // lane l finishes output (i, j) with i * NPW + j == l
+    int mine = 0;
+#pragma unroll
+    for (int i = 0; i < MB; ++i)
+#pragma unroll
+        for (int j = 0; j < NPW; ++j)
+            if (lane == i * NPW + j) mine = acc[i][j];
+    if (lane < MB * NPW) {
+        const int m = m0 + lane / NPW, n = n0 + lane % NPW;
+        if (m < M && n < N) {
+            if (raw_i32) {
+                static_cast<int32_t*>(out)[static_cast<int64_t>(m) * ldo + n] = mine;
+            } else {
+                float t = __int2float_rn(mine);
+                t = __fmul_rn(t, s_tok[m]);
+                t = __fmul_rn(t, s_ch[n]);
+                if (bias != nullptr) t = __fadd_rn(t, bias[n]);
+                static_cast<__nv_bfloat16*>(out)[static_cast<int64_t>(m) * ldo + n] = __float2bfloat16_rn(t);
+            }
+        }
+    }
+}
+
+template <int MB, int NPW, int WARPS>
+cudaError_t launch(const GemmArgs& a, cudaStream_t st) {
+    dim3 grid((a.N + WARPS * NPW - 1) / (WARPS * NPW), (a.M + MB - 1) / MB);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(WARPS * 32);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = a.after_quantizer ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, gemm_simt_kernel<MB, NPW, WARPS>, a.qa, a.lda_q, a.s_tok, a.qw, a.s_ch, a.bias,
+                              a.out, a.ldo, a.M, a.N, a.K, a.raw_i32 ? 1 : 0, a.after_quantizer ? 1 : 0);
+}
+
+} // namespace
+
+cudaError_t launch_gemm_simt(const GemmArgs& a, cudaStream_t st) {
+    if (a.M <= 2) return launch<2, 4, 4>(a, st);
+    if (a.M <= 4) return launch<4, 4, 4>(a, st);
+    return launch<8, 4, 4>(a, st);
+}
+
+} // namespace w8a8

@@ -10,3 +10,6 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200, sm_100a)")
+    # the CUDA library and the oracle are built in-tree on first use (nvcc cross-compiles without a GPU)
+    import __graft_entry__
+    __graft_entry__.build()

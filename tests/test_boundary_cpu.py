@@ -1,0 +1,102 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every symbol the
+header declares, sizes workspaces as documented, and rejects bad arguments before touching CUDA."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2606_14598_b200 as w8
+from paper_2606_14598_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "w8a8_linear.h")
+
+
+def declared_functions():
+    src = open(HEADER).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    return sorted(set(re.findall(r"\b(int8_[a-z0-9_]+)\s*\(", src)))
+
+
+def test_library_exports_every_declared_symbol():
+    names = declared_functions()
+    assert len(names) >= 10
+    lib = ctypes.CDLL(binding.LIB_PATH)
+    for n in names:
+        assert hasattr(lib, n), n
+    assert sorted(binding.EXPORTS) == names
+
+
+def test_status_strings():
+    for code in range(8):
+        assert w8.status_string(code) and w8.status_string(code) != "unknown status"
+    assert w8.status_string(99) == "unknown status"
+
+
+def test_workspace_sizes():
+    assert w8.int8_linear_workspace_bytes(4608, 3072, 12288, w8.ACT_INT8) == 256
+    s_off, q_off = w8.int8_linear_workspace_offsets(4608, 12288)
+    assert s_off == 256 and q_off == 256 + 4608 * 4 and q_off % 256 == 0
+    assert w8.int8_linear_workspace_bytes(4608, 3072, 12288, w8.ACT_BF16) == q_off + 4608 * 12288
+    s_off, q_off = w8.int8_linear_workspace_offsets(2, 3072)
+    assert q_off == 512 and w8.int8_linear_workspace_bytes(2, 8, 3072, w8.ACT_BF16) == 512 + 6144
+    assert w8.int8_linear_workspace_bytes(0, 8, 16) == 0
+    assert w8.int8_linear_workspace_bytes(8, 8, 16, 5) == 0
+
+
+def test_configs_are_listed():
+    n = w8.num_configs()
+    assert n >= 2 and all(w8.config_name(i) for i in range(n)) and w8.config_name(n) is None
+    assert w8.force_config(-1) == -1
+
+
+# fake, well-aligned addresses: argument checks run before any CUDA call, so nothing is dereferenced
+P = 0x10000
+
+
+def fused(A=P, a_dtype=0, lda=64, s_tok=None, qw=P, s_ch=P, bias=None, out=P, ldo=64, M=32, N=64, K=64, ws=P, ws_bytes=1 << 20):
+    return binding.raw().int8_linear_fused(A, a_dtype, lda, s_tok, qw, s_ch, bias, out, ldo, M, N, K, ws, ws_bytes, None)
+
+
+def test_fused_rejects_bad_arguments_before_any_launch():
+    INVALID, ALIGN, KOVF, WS = 1, 2, 3, 4
+    assert fused(A=None) == INVALID
+    assert fused(qw=None) == INVALID and fused(s_ch=None) == INVALID and fused(out=None) == INVALID
+    assert fused(a_dtype=2) == INVALID
+    assert fused(a_dtype=1, s_tok=None) == INVALID          # int8 activations need their scales
+    assert fused(a_dtype=0, s_tok=P) == INVALID             # bf16 activations must not bring scales
+    assert fused(M=0) == INVALID and fused(N=-8) == INVALID and fused(K=0) == INVALID
+    assert fused(lda=32) == INVALID and fused(ldo=56) == INVALID
+    assert fused(K=133152, lda=133152) == KOVF
+    assert fused(K=w8.K_MAX + 8, lda=w8.K_MAX + 8) == KOVF
+    assert fused(K=72, lda=72) == ALIGN                     # K % 16
+    assert fused(N=60, ldo=64) == ALIGN                     # N % 8
+    assert fused(ldo=68) == ALIGN
+    assert fused(a_dtype=1, s_tok=P, lda=72) == ALIGN       # int8 row stride not a multiple of 16 bytes
+    assert fused(A=P + 8) == ALIGN and fused(qw=P + 4) == ALIGN and fused(out=P + 2) == ALIGN
+    assert fused(ws=None) == WS and fused(ws=P + 128) == WS and fused(ws_bytes=255) == WS
+    need = w8.int8_linear_workspace_bytes(32, 64, 64, 0)
+    assert fused(ws_bytes=need - 1) == WS
+
+
+def test_quantizers_reject_bad_arguments():
+    lib = binding.raw()
+    assert lib.int8_quantize_weight_per_channel(None, 8, 16, 16, P, P, None) == 1
+    assert lib.int8_quantize_weight_per_channel(P, 8, 16, 8, P, P, None) == 1      # ldw < K
+    assert lib.int8_quantize_weight_per_channel(P, 8, 24, 24, P, P, None) == 2     # K % 16
+    assert lib.int8_quantize_weight_per_channel(P + 4, 8, 16, 16, P, P, None) == 2
+    assert lib.int8_quantize_act_per_token(P, 0, 16, 16, P, P, None) == 1
+    assert lib.int8_quantize_act_per_token(P, 8, 16, 20, P, P, None) == 2          # lda % 8
+    assert lib.int8_gemm_i32_debug(P, P, None, 8, 8, 16, P, 256, None) == 1
+    assert lib.int8_gemm_i32_debug(P, P, P, 8, 6, 16, P, 256, None) == 2
+    assert lib.int8_gemm_i32_debug(P, P, P, 8, 8, 16, P, 8, None) == 4
+    assert lib.int8_check_status(None, None) == 4
+
+
+def test_no_device_means_a_loud_error_not_a_fallback():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    # valid arguments, no device: the call must fail (CUDA error), never compute on the CPU
+    assert fused() in (5, 6)

@@ -1,0 +1,317 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle, element by element.
+
+Bars: int8 codes, fp32 scales and int32 accumulators bit-exact; bf16 outputs within 1 bf16 ulp
+(ordered-integer distance of the bit patterns, +0 == -0) with cosine >= 0.99999. Because the
+kernels follow the oracle's operation order, the bf16 outputs are in fact expected to be equal
+bit for bit, and the tests assert that too.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2606_14598_b200 as w8
+from paper_2606_14598_b200 import inputs as synth
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+def n_tc_configs():
+    return w8.num_configs() - 1          # the last configuration is the CUDA-core path
+
+
+@pytest.fixture(autouse=True)
+def _reset_config():
+    w8.force_config(-1)
+    yield
+    w8.force_config(-1)
+
+
+def ordered(bits):
+    b = bits.astype(np.int32)
+    return np.where(b & 0x8000, -(b & 0x7FFF), b)
+
+
+def bits_f64(bits):
+    return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def assert_bf16_close(got_bits, ref_bits, exact=True):
+    assert got_bits.shape == ref_bits.shape
+    d = np.abs(ordered(got_bits) - ordered(ref_bits))
+    assert d.max() <= 1, f"max ulp distance {d.max()} at {np.unravel_index(d.argmax(), d.shape)}"
+    g, r = bits_f64(got_bits).ravel(), bits_f64(ref_bits).ravel()
+    assert np.isfinite(g).all()
+    nz = r != 0
+    if nz.any():
+        rel = np.abs(g[nz] - r[nz]) / np.abs(r[nz])
+        assert rel.max() <= 2.0 ** -7
+    den = np.sqrt((g * g).sum() * (r * r).sum())
+    if den > 0:
+        assert (g * r).sum() / den >= 0.99999
+    if exact:
+        assert (d == 0).all(), f"{int((d != 0).sum())} of {d.size} outputs differ by one ulp"
+
+
+def check_status(ws):
+    st = w8.int8_check_status(ws)
+    assert st == 0, w8.status_string(st)
+
+
+def rand_codes(rng, shape, lo=-127):
+    return rng.integers(lo, 128, shape, dtype=np.int8)
+
+
+# ------------------------------------------------------------------------------- quantizers (T1)
+
+@pytest.mark.parametrize("M,K", [(1, 16), (7, 48), (33, 2048), (300, 3072), (9, 4096), (5, 8192), (40, 12288),
+                                 (3, 16384), (3, 16400), (2, 40000)])
+def test_act_quantizer_bit_exact(M, K):
+    spec = synth.LinearSpec(f"q{M}x{K}", M, K, 8, outlier_frac=0.01 if K >= 256 else 0.0)
+    A = synth.make_activations(spec)
+    if M > 2:
+        A[1] = 0                                   # an all-zero token
+    qa_ref, s_ref = oracle.quantize_act_per_token(synth.bf16_bits(A))
+    qa, s = w8.int8_quantize_act_per_token(A.to(DEV))
+    assert np.array_equal(s.cpu().numpy().view(np.uint32), s_ref.view(np.uint32))
+    assert np.array_equal(qa.cpu().numpy(), qa_ref)
+
+
+def test_act_quantizer_gelu_rows_and_row_stride():
+    spec = synth.LinearSpec("qg", 70, 1024, 8, act="gelu", outlier_frac=0.0)
+    A = synth.make_activations(spec)
+    qa_ref, s_ref = oracle.quantize_act_per_token(synth.bf16_bits(A))
+    wide = torch.full((70, 1024 + 64), 7.0, dtype=torch.bfloat16, device=DEV)
+    wide[:, :1024] = A.to(DEV)
+    qa, s = w8.int8_quantize_act_per_token(wide[:, :1024])           # lda = 1088
+    assert np.array_equal(s.cpu().numpy(), s_ref) and np.array_equal(qa.cpu().numpy(), qa_ref)
+
+
+def test_act_quantizer_hand_ties_on_device():
+    x = torch.tensor([[127, 0.5, 1.5, 2.5, -0.5, -1.5, -2.5, 63.5, 126.5, -126.5, 0.375, 0.625, -127, 3, 0, 0]],
+                     dtype=torch.bfloat16)
+    qa, s = w8.int8_quantize_act_per_token(x.to(DEV))
+    assert s.item() == 1.0
+    assert qa.cpu().tolist() == [[127, 0, 2, 2, 0, -2, -2, 64, 126, -126, 0, 1, -127, 3, 0, 0]]
+
+
+@pytest.mark.parametrize("N,K", [(5, 16), (256, 256), (100, 3072), (17, 12288), (3, 16400)])
+def test_weight_quantizer_bit_exact(N, K):
+    spec = synth.LinearSpec(f"w{N}x{K}", 8, K, N)
+    W = synth.make_weight(spec)
+    if N > 2:
+        W[2] = 0
+    qw_ref, s_ref = oracle.quantize_weight_per_channel(W.numpy())
+    qw, s = w8.int8_quantize_weight_per_channel(W.to(DEV))
+    assert np.array_equal(s.cpu().numpy().view(np.uint32), s_ref.view(np.uint32))
+    assert np.array_equal(qw.cpu().numpy(), qw_ref)
+
+
+# ------------------------------------------------------------------------------- raw accumulators (T2)
+
+ACC_SHAPES = [
+    (128, 256, 128),     # exactly one tile, one k-block
+    (128, 256, 16), (128, 256, 32), (128, 256, 48), (128, 256, 144), (128, 128, 400),
+    (1, 8, 16), (17, 8, 64), (129, 264, 160),
+    (300, 328, 384),     # ragged in M and N, several tiles
+    (640, 10240, 256),   # 200 tiles of 128x256: more than one tile per CTA, both accumulator buffers
+    (2816, 3072, 512),
+]
+
+
+@pytest.mark.parametrize("M,N,K", ACC_SHAPES)
+def test_accumulators_bit_exact_all_tensor_core_configs(M, N, K):
+    rng = np.random.default_rng(M * 7 + N * 3 + K)
+    qa, qw = rand_codes(rng, (M, K)), rand_codes(rng, (N, K))
+    ref = oracle.gemm_i32(qa, qw)
+    dqa, dqw = torch.from_numpy(qa).to(DEV), torch.from_numpy(qw).to(DEV)
+    for cfg in range(w8.num_configs()):
+        if cfg == n_tc_configs() and M * N * K > 2 ** 31:
+            continue                                    # the CUDA-core path is slow on big shapes
+        w8.force_config(cfg)
+        ws = w8.alloc_workspace(M, N, K, w8.ACT_INT8, DEV)
+        acc = w8.int8_gemm_i32_debug(dqa, dqw, ws)
+        check_status(ws)
+        assert np.array_equal(acc.cpu().numpy(), ref), f"config {cfg}: {w8.config_name(cfg)}"
+
+
+def test_accumulators_overflow_edge_and_minus_128():
+    # K * 127^2 just below 2^31, every product at its extreme
+    K = 133136
+    qa = np.full((130, K), 127, np.int8)
+    qa[1::2] = -127
+    qw = np.full((16, K), 127, np.int8)
+    qw[3] = -127
+    dqa, dqw = torch.from_numpy(qa).to(DEV), torch.from_numpy(qw).to(DEV)
+    want = (qa[:, :1].astype(np.int64) * qw[:, :1].astype(np.int64).T) * K
+    assert abs(want).max() == K * 16129 < 2 ** 31
+    for cfg in range(n_tc_configs()):
+        w8.force_config(cfg)
+        acc = w8.int8_gemm_i32_debug(dqa, dqw)
+        assert np.array_equal(acc.cpu().numpy().astype(np.int64), want), cfg
+    # -128 codes are tolerated and exact while K <= 131071
+    w8.force_config(-1)
+    rng = np.random.default_rng(3)
+    qa2, qw2 = rand_codes(rng, (200, 512), lo=-128), rand_codes(rng, (264, 512), lo=-128)
+    qa2[0, :] = -128
+    qw2[0, :] = -128
+    acc = w8.int8_gemm_i32_debug(torch.from_numpy(qa2).to(DEV), torch.from_numpy(qw2).to(DEV))
+    assert np.array_equal(acc.cpu().numpy(), oracle.gemm_i32(qa2, qw2))
+    assert acc[0, 0].item() == 512 * 16384
+
+
+def test_accumulators_match_library_int_mm():
+    # the paper's own gate: the integer accumulation equals an independent integer matmul
+    rng = np.random.default_rng(8)
+    qa = torch.from_numpy(rand_codes(rng, (2816, 3072))).to(DEV)
+    qw = torch.from_numpy(rand_codes(rng, (3072, 3072))).to(DEV)
+    want = torch._int_mm(qa, qw.t())
+    for cfg in range(n_tc_configs()):
+        w8.force_config(cfg)
+        assert torch.equal(w8.int8_gemm_i32_debug(qa, qw), want), cfg
+
+
+# ------------------------------------------------------------------------------- fused output (T3)
+
+FUSED_SHAPES = [(128, 256, 256), (300, 384, 328), (129, 3072, 264), (1000, 1024, 1536), (640, 256, 10240)]
+
+
+@pytest.mark.parametrize("M,K,N", FUSED_SHAPES)
+@pytest.mark.parametrize("use_bias", [True, False])
+def test_fused_from_bf16_matches_oracle(M, K, N, use_bias):
+    spec = synth.LinearSpec(f"f{M}x{K}x{N}", M, K, N, bias=use_bias)
+    t = synth.make_linear(spec)
+    if M > 4:
+        t["A"][3] = 0                                   # zero token: output row equals the bias
+    qw_ref, s_ch_ref = oracle.quantize_weight_per_channel(t["W"].numpy())
+    bias_np = t["bias"].numpy() if use_bias else None
+    ref = oracle.linear_fused_bf16(synth.bf16_bits(t["A"]), qw_ref, s_ch_ref, bias_np)
+    qw, s_ch = w8.int8_quantize_weight_per_channel(t["W"].to(DEV))
+    assert np.array_equal(qw.cpu().numpy(), qw_ref) and np.array_equal(s_ch.cpu().numpy(), s_ch_ref)
+    bias = t["bias"].to(DEV) if use_bias else None
+    A = t["A"].to(DEV)
+    for cfg in range(w8.num_configs()):
+        w8.force_config(cfg)
+        ws = w8.alloc_workspace(M, N, K, w8.ACT_BF16, DEV)
+        out = w8.int8_linear_fused(A, qw, s_ch, bias, workspace=ws)
+        check_status(ws)
+        # the intermediate tensors the call leaves in the workspace
+        s_off, q_off = w8.int8_linear_workspace_offsets(M, K)
+        s_tok = ws[s_off:s_off + 4 * M].view(torch.float32).cpu().numpy()
+        qa = ws[q_off:q_off + M * K].view(torch.int8).view(M, K).cpu().numpy()
+        assert np.array_equal(s_tok, ref["s_tok"]) and np.array_equal(qa, ref["qa"]), cfg
+        assert_bf16_close(synth.bf16_bits(out.cpu()), ref["out"])
+    if M > 4 and use_bias:
+        zero_row = synth.bf16_bits(out.cpu())[3]
+        assert np.array_equal(zero_row, synth.bf16_bits(t["bias"].to(torch.bfloat16)))
+
+
+def test_fused_from_int8_with_row_stride_and_guard_bands():
+    M, K, N = 200, 512, 328
+    rng = np.random.default_rng(21)
+    qa, qw = rand_codes(rng, (M, K)), rand_codes(rng, (N, K))
+    s_tok = (rng.random(M) * 0.05 + 0.01).astype(np.float32)
+    s_ch = (rng.random(N) * 0.0008 + 0.0002).astype(np.float32)
+    bias = (rng.standard_normal(N) * 0.01).astype(np.float32)
+    ref = oracle.linear_fused_int8(qa, s_tok, qw, s_ch, bias)
+    qa_wide = torch.zeros((M, K + 64), dtype=torch.int8, device=DEV)
+    qa_wide[:, :K] = torch.from_numpy(qa).to(DEV)
+    SENT = -2.0
+    canvas = torch.full((M + 40, N + 56), SENT, dtype=torch.bfloat16, device=DEV)   # output lives inside a larger buffer
+    for cfg in range(w8.num_configs()):
+        w8.force_config(cfg)
+        canvas.fill_(SENT)
+        out_view = canvas[8:8 + M, 16:16 + N]
+        ws = w8.alloc_workspace(M, N, K, w8.ACT_INT8, DEV)
+        w8.int8_linear_fused(qa_wide[:, :K], torch.from_numpy(qw).to(DEV), torch.from_numpy(s_ch).to(DEV),
+                             torch.from_numpy(bias).to(DEV), s_tok=torch.from_numpy(s_tok).to(DEV), out=out_view,
+                             workspace=ws)
+        check_status(ws)
+        assert_bf16_close(synth.bf16_bits(out_view.contiguous().cpu()), ref["out"])
+        mask = torch.ones_like(canvas, dtype=torch.bool)
+        mask[8:8 + M, 16:16 + N] = False
+        assert (canvas[mask] == SENT).all(), f"config {cfg} wrote outside its output"
+
+
+@pytest.mark.parametrize("M", [1, 2, 5, 16])
+def test_skinny_m_path(M):
+    spec = synth.LinearSpec(f"skinny{M}", M, 3072, 2048, outlier_frac=0.0)
+    t = synth.make_linear(spec)
+    qw_ref, s_ch_ref = oracle.quantize_weight_per_channel(t["W"].numpy())
+    ref = oracle.linear_fused_bf16(synth.bf16_bits(t["A"]), qw_ref, s_ch_ref, t["bias"].numpy())
+    qw, s_ch = w8.int8_quantize_weight_per_channel(t["W"].to(DEV))
+    ws = w8.alloc_workspace(M, spec.N, spec.K, w8.ACT_BF16, DEV)
+    out = w8.int8_linear_fused(t["A"].to(DEV), qw, s_ch, t["bias"].to(DEV), workspace=ws)
+    check_status(ws)
+    assert_bf16_close(synth.bf16_bits(out.cpu()), ref["out"])
+
+
+def test_run_to_run_identical_and_host_buffer_entry_point():
+    spec = synth.LinearSpec("rr", 1100, 1024, 1544)
+    t = synth.make_linear(spec)
+    qw, s_ch = w8.int8_quantize_weight_per_channel(t["W"].to(DEV))
+    A, bias = t["A"].to(DEV), t["bias"].to(DEV)
+    ws = w8.alloc_workspace(spec.M, spec.N, spec.K, w8.ACT_BF16, DEV)
+    first = w8.int8_linear_fused(A, qw, s_ch, bias, workspace=ws).clone()
+    for _ in range(5):
+        assert torch.equal(w8.int8_linear_fused(A, qw, s_ch, bias, workspace=ws), first)
+    check_status(ws)
+    A_host = t["A"].pin_memory()
+    out_host = torch.empty((spec.M, spec.N), dtype=torch.bfloat16).pin_memory()
+    d_A, d_out = torch.empty_like(A), torch.empty_like(first)
+    w8.int8_linear_fused_host(A_host, d_A, qw, s_ch, bias, d_out, out_host, ws)
+    check_status(ws)
+    assert torch.equal(out_host, first.cpu())
+
+
+# ------------------------------------------------------------------------------- benchmark configs, full size (T4)
+
+def sample_rows(M, n=48):
+    """Rows spread over every part of the M range, including both ends of the first and last tiles."""
+    fixed = [0, 1, 31, 32, 127, 128, M - 129, M - 128, M - 2, M - 1]
+    rng = np.random.default_rng(M)
+    extra = rng.integers(0, M, n).tolist()
+    return np.array(sorted({r for r in fixed + extra if 0 <= r < M}), dtype=np.int64)
+
+
+ALL_SPECS = [s for name in ("c1", "c2", "c3", "c4", "c5") for s in synth.CONFIGS[name]]
+
+
+@pytest.mark.parametrize("spec", ALL_SPECS, ids=[s.name for s in ALL_SPECS])
+def test_benchmark_configs_full_size(spec):
+    """The launch configuration bench.py times (automatic config, from bf16), at full size. The oracle
+    recomputes a sample of whole output rows (every column of them); all int8 codes and scales of
+    those rows, their int32 accumulators and their bf16 outputs must match. The full accumulator
+    matrix is also compared with the library integer matmul."""
+    t = synth.make_linear(spec)
+    M, K, N = spec.M, spec.K, spec.N
+    qw_ref, s_ch_ref = oracle.quantize_weight_per_channel(t["W"].numpy())
+    qw, s_ch = w8.int8_quantize_weight_per_channel(t["W"].to(DEV))
+    assert np.array_equal(qw.cpu().numpy(), qw_ref) and np.array_equal(s_ch.cpu().numpy(), s_ch_ref)
+    A, bias = t["A"].to(DEV), t["bias"].to(DEV)
+    ws = w8.alloc_workspace(M, N, K, w8.ACT_BF16, DEV)
+    out = w8.int8_linear_fused(A, qw, s_ch, bias, workspace=ws)
+    check_status(ws)
+    assert torch.isfinite(out.float()).all()
+    rows = sample_rows(M) if M > 256 else np.arange(M)
+    A_rows = np.ascontiguousarray(synth.bf16_bits(t["A"])[rows])
+    ref = oracle.linear_fused_bf16(A_rows, qw_ref, s_ch_ref, t["bias"].numpy())
+    s_off, q_off = w8.int8_linear_workspace_offsets(M, K)
+    s_tok = ws[s_off:s_off + 4 * M].view(torch.float32)
+    qa = ws[q_off:q_off + M * K].view(torch.int8).view(M, K)
+    ridx = torch.from_numpy(rows).to(DEV)
+    assert np.array_equal(s_tok[ridx].cpu().numpy(), ref["s_tok"])
+    assert np.array_equal(qa[ridx].cpu().numpy(), ref["qa"])
+    assert_bf16_close(synth.bf16_bits(out[ridx].cpu()), ref["out"])
+    # raw accumulators: sampled rows vs the oracle, everything vs the library integer matmul
+    acc = w8.int8_gemm_i32_debug(qa, qw)
+    assert np.array_equal(acc[ridx].cpu().numpy(), ref["acc"])
+    if M > 16:
+        assert torch.equal(acc, torch._int_mm(qa, qw.t()))
+    # pre-quantized entry gives the same bits as the from-bf16 entry
+    ws2 = w8.alloc_workspace(M, N, K, w8.ACT_INT8, DEV)
+    out2 = w8.int8_linear_fused(qa, qw, s_ch, bias, s_tok=s_tok, workspace=ws2)
+    check_status(ws2)
+    assert torch.equal(out2, out)
