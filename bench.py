@@ -1,0 +1,398 @@
+#!/usr/bin/env python
+"""Benchmark of the fused W8A8 linear on seeded synthetic DiT-shaped inputs.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c4] [--impl reference]
+
+One step = one pass of the whole hot path (per-token quantization of the bf16 activations, int8
+tensor-core GEMM, dequantizing epilogue) over every linear of the workload; the default workload
+is the MLP up and down projections at 1024px (M=4608, 3072 -> 12288 -> 3072), the shapes the
+throughput target is quoted on. Prints ONE JSON line on stdout (diagnostics go to stderr).
+
+`--impl reference` times the CPU oracle, as it stands, on the host cores on a bounded sample of
+the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "fused W8A8 linear TOPS (% of B200 dense INT8 peak) per DiT GEMM shape"
+INT8_PEAK_TOPS = 4500.0            # B200 datasheet, dense INT8
+L2_BYTES = 126 * 1024 * 1024
+
+
+def log(*a):
+    print(*a, file=sys.stderr, flush=True)
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------------------ clocks
+
+class ClockSampler:
+    """Samples SM clock, power and clock-event reasons through NVML while the timed region runs."""
+
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap",
+               0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting", 0x100: "display_clock_setting",
+               0x10: "sync_boost"}
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.period = period_s
+        self.samples, self.power, self.reasons = [], [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thr = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            visible = os.environ.get("CUDA_VISIBLE_DEVICES")
+            if visible:
+                ids = [v for v in visible.split(",") if v.strip() != ""]
+                tok = ids[index] if index < len(ids) else ids[0]
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(int(tok)) if tok.isdigit() else pynvml.nvmlDeviceGetHandleByUUID(tok)
+            else:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception as e:          # NVML missing: report that no clocks were sampled
+            log(f"[bench] NVML unavailable: {e}")
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(float(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                self.power.append(nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0)
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thr = threading.Thread(target=self._loop, daemon=True)
+            self._thr.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thr is not None:
+            self._thr.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["not sampled"], "samples": 0}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples),
+                "power_w_max": max(self.power) if self.power else None}
+
+
+# ------------------------------------------------------------------------------------------ reference arm
+
+def reference_sample_rows(spec, target_gmac=40.0):
+    """Rows of one linear the oracle recomputes per step, sized for a few seconds of CPU work."""
+    rows = int(target_gmac * 1e9 / (spec.K * spec.N))
+    return max(1, min(spec.M, rows))
+
+
+def time_oracle(specs, steps, warmup, target_gmac):
+    """Times the oracle (quantize + integer GEMM + epilogue) on the first rows of each linear."""
+    import numpy as np
+
+    import oracle
+    from paper_2606_14598_b200 import inputs as synth
+
+    prepared = []
+    for spec in specs:
+        rows = reference_sample_rows(spec, target_gmac)
+        A = synth.bf16_bits(synth.make_activations(spec, rows=slice(0, rows)))
+        qw, s_ch = oracle.quantize_weight_per_channel(synth.make_weight(spec).numpy())
+        bias = synth.make_bias(spec)
+        prepared.append((spec, rows, np.ascontiguousarray(A), qw, s_ch, None if bias is None else bias.numpy()))
+    ops = sum(2.0 * rows * s.N * s.K for s, rows, *_ in prepared)
+    times = []
+    for i in range(warmup + steps):
+        t0 = time.perf_counter()
+        for _, _, A, qw, s_ch, bias in prepared:
+            oracle.linear_fused_bf16(A, qw, s_ch, bias)
+        dt = time.perf_counter() - t0
+        if i >= warmup:
+            times.append(dt)
+    sec = sum(times) / len(times)
+    sample = ", ".join(f"{s.name}: first {rows} of {s.M} rows" for s, rows, *_ in prepared)
+    return ops / sec / 1e12, sec, oracle.num_threads(), sample
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2606_14598_b200 import inputs as synth
+    specs = synth.CONFIGS[args.workload]
+    steps, warmup = max(1, min(args.steps, 3)), min(args.warmup, 1)
+    tops, sec, cores, sample = time_oracle(specs, steps, warmup, target_gmac=20.0)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": tops, "unit": "TOPS", "n_gpus": args.gpus,
+        "steps": steps, "warmup": warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {"workload": workload_name(args.workload, specs), "sample": sample},
+        "pct_of_int8_peak": 100.0 * tops / INT8_PEAK_TOPS,
+        "cpu_baseline": {"value": tops, "unit": "TOPS", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": tops, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_name(key, specs):
+    return f"{key}: " + " + ".join(f"{s.name} (M={s.M}, K={s.K}, N={s.N})" for s in specs)
+
+
+# ------------------------------------------------------------------------------------------ CUDA arm
+
+def cuda_timer(torch, fn, iters, warm):
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(iters)]
+    for a, b in ev:
+        a.record()
+        fn()
+        b.record()
+    torch.cuda.synchronize()
+    return [a.elapsed_time(b) * 1e-3 for a, b in ev]
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--workload", default="c4", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--sets", type=int, default=3, help="rotating input/weight sets (keeps steps out of L2)")
+    ap.add_argument("--no-extras", action="store_true", help="skip e2e, context and CPU-baseline legs")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+
+    import paper_2606_14598_b200 as w8
+    from paper_2606_14598_b200 import dist as wdist
+    from paper_2606_14598_b200 import inputs as synth
+    from paper_2606_14598_b200 import roofline as model
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the CUDA path has no CPU fallback (use --impl reference)")
+    args.warmup = max(args.warmup, 3)
+    rank, local_rank, world = wdist.init("nccl")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    specs = synth.CONFIGS[args.workload]
+    peaks = measured_peaks()
+
+    # ---- set-up (untimed): seeded inputs, weights quantized on the device by the library
+    sets = []
+    for r in range(args.sets):
+        layer = []
+        for spec in specs:
+            seed = 1000 * rank + r
+            A = synth.make_activations(spec, seed).to(dev)
+            qw, s_ch = w8.int8_quantize_weight_per_channel(synth.make_weight(spec, seed).to(dev))
+            bias = synth.make_bias(spec, seed)
+            layer.append({"spec": spec, "A": A, "qw": qw, "s_ch": s_ch, "bias": None if bias is None else bias.to(dev),
+                          "out": torch.empty((spec.M, spec.N), dtype=torch.bfloat16, device=dev),
+                          "ws": w8.alloc_workspace(spec.M, spec.N, spec.K, w8.ACT_BF16, dev)})
+        sets.append(layer)
+    torch.cuda.synchronize()
+    set_bytes = sum(model.bytes_from_bf16(s.M, s.N, s.K) for s in specs)
+    ops_per_step = float(sum(s.ops for s in specs))
+
+    def step(i):
+        for L in sets[i % len(sets)]:
+            w8.int8_linear_fused(L["A"], L["qw"], L["s_ch"], L["bias"], out=L["out"], workspace=L["ws"])
+
+    # ---- health gate: the GPU must deliver its usual bf16 rate, or the numbers below mean nothing
+    health = None
+    if rank == 0 and not args.no_extras:
+        a = torch.randn(8192, 8192, device=dev, dtype=torch.bfloat16)
+        b = torch.randn(8192, 8192, device=dev, dtype=torch.bfloat16)
+        ts = cuda_timer(torch, lambda: torch.matmul(a, b), 10, 3)
+        tf = 2 * 8192 ** 3 / min(ts) / 1e12
+        health = {"bf16_matmul_tflops": tf, "ok": tf >= 0.8 * peaks["bf16_tflops"]}
+        del a, b
+
+    # ---- the timed region
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    wdist.barrier(dev)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local_rank) as clocks:
+        e0.record()
+        for i in range(args.steps):
+            step(i)
+        e1.record()
+        torch.cuda.synchronize()
+    wdist.barrier(dev)
+    sec_local = e0.elapsed_time(e1) * 1e-3
+    for layer in sets:
+        for L in layer:
+            st = w8.int8_check_status(L["ws"])
+            if st != 0:
+                raise SystemExit(f"device-side status: {w8.status_string(st)}")
+    ops_total_per_sec, sec = wdist.aggregate_throughput(ops_per_step * args.steps, sec_local, dev)
+    tops = ops_total_per_sec / 1e12
+    launches = args.steps * sum(2 for _ in specs)      # quantizer + GEMM per linear
+
+    line = {
+        "metric": METRIC, "value": tops, "unit": "TOPS", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": sec / args.steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int8", "data": "synthetic",
+        "config": {"workload": workload_name(args.workload, specs), "entry": "int8_linear_fused from bf16 activations",
+                   "l2": f"inputs larger than L2: {len(sets)} rotating sets of {set_bytes / 1e6:.0f} MB each",
+                   "parallelism": f"dp{world} over tokens, weights replicated, no collective"},
+        "pct_of_int8_peak": 100.0 * tops / (INT8_PEAK_TOPS * world), "int8_peak_tops": INT8_PEAK_TOPS,
+        "clocks": clocks.summary(), "gpu_launches": launches,
+    }
+
+    if rank == 0:
+        # ---- per-kernel timing (same kernels, same launch configuration, timed one by one)
+        per_shape, gemm_ops, gemm_sec, q_bytes, q_sec = [], 0.0, 0.0, 0.0, 0.0
+        for j, spec in enumerate(specs):
+            M, K, N = spec.M, spec.K, spec.N
+            s_off, q_off = w8.int8_linear_workspace_offsets(M, K)
+            rot = [sets[r][j] for r in range(len(sets))]
+            views = [(L, L["ws"][s_off:s_off + 4 * M].view(torch.float32), L["ws"][q_off:q_off + M * K].view(torch.int8).view(M, K))
+                     for L in rot]
+            ws8 = w8.alloc_workspace(M, N, K, w8.ACT_INT8, dev)
+            it = [0]
+
+            def gemm_only():
+                L, s_tok, qa = views[it[0] % len(views)]
+                it[0] += 1
+                w8.int8_linear_fused(qa, L["qw"], L["s_ch"], L["bias"], s_tok=s_tok, out=L["out"], workspace=ws8)
+
+            def quant_only():
+                L, s_tok, qa = views[it[0] % len(views)]
+                it[0] += 1
+                w8.int8_quantize_act_per_token(L["A"], qa, s_tok)
+
+            def fused():
+                L, _, _ = views[it[0] % len(views)]
+                it[0] += 1
+                w8.int8_linear_fused(L["A"], L["qw"], L["s_ch"], L["bias"], out=L["out"], workspace=L["ws"])
+
+            n_it = 30
+            tg = statistics.mean(cuda_timer(torch, gemm_only, n_it, 5))
+            tq = statistics.mean(cuda_timer(torch, quant_only, n_it, 5))
+            tf_ = statistics.mean(cuda_timer(torch, fused, n_it, 5))
+            per_shape.append({"name": spec.name, "M": M, "K": K, "N": N,
+                              "fused_from_bf16_us": tf_ * 1e6, "fused_from_bf16_tops": spec.ops / tf_ / 1e12,
+                              "pct_of_int8_peak": 100.0 * spec.ops / tf_ / 1e12 / INT8_PEAK_TOPS,
+                              "gemm_epilogue_us": tg * 1e6, "gemm_epilogue_tops": spec.ops / tg / 1e12,
+                              "quantizer_us": tq * 1e6, "quantizer_gbs": model.quantizer_bytes(M, K) / tq / 1e9})
+            if M > 16:
+                gemm_ops += spec.ops
+                gemm_sec += tg
+            q_bytes += model.quantizer_bytes(M, K)
+            q_sec += tq
+        line["per_shape"] = per_shape
+        int8_peak_measured = 2.0 * peaks["bf16_tflops_sustained"]
+        achieved = gemm_ops / gemm_sec / 1e12 if gemm_sec > 0 else 0.0
+        line["roofline"] = {
+            "kernel": "gemm_tc_kernel (tcgen05.mma.kind::i8 + dequant epilogue)", "bound": "tensor",
+            "achieved": achieved, "peak": int8_peak_measured, "unit": "TFLOP/s", "frac": achieved / int8_peak_measured,
+            "traffic": None,
+            "peak_source": f"2 x {peaks['source']} sustained bf16 cuBLAS rate ({peaks['bf16_tflops_sustained']} TFLOP/s); "
+                           "int8 multiply-add counted as 2 ops",
+            "quantizer": {"bound": "hbm", "achieved": q_bytes / q_sec / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                          "frac": q_bytes / q_sec / 1e9 / peaks["hbm_gbs"]},
+        }
+        if health is not None:
+            line["health"] = health
+
+        if not args.no_extras:
+            # ---- end to end through the host-buffer entry point: pinned host activations in, host result out
+            e2e_sets = []
+            for L in sets[0]:
+                spec = L["spec"]
+                e2e_sets.append({"L": L, "A_host": L["A"].cpu().pin_memory(),
+                                 "out_host": torch.empty((spec.M, spec.N), dtype=torch.bfloat16).pin_memory(),
+                                 "d_A": torch.empty_like(L["A"])})
+
+            def e2e_step():
+                for e in e2e_sets:
+                    L = e["L"]
+                    w8.int8_linear_fused_host(e["A_host"], e["d_A"], L["qw"], L["s_ch"], L["bias"], L["out"], e["out_host"], L["ws"])
+
+            n_e2e = 10
+            for _ in range(3):
+                e2e_step()
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            t0 = time.perf_counter()
+            a.record()
+            for _ in range(n_e2e):
+                e2e_step()
+            b.record()
+            torch.cuda.synchronize()
+            wall = time.perf_counter() - t0
+            e2e_sec = max(a.elapsed_time(b) * 1e-3, wall) / n_e2e
+            line["e2e"] = {"value": ops_per_step / e2e_sec / 1e12, "unit": "TOPS",
+                           "h2d_bytes_per_step": sum(2 * s.M * s.K for s in specs),
+                           "d2h_bytes_per_step": sum(2 * s.M * s.N for s in specs), "ms_per_step": e2e_sec * 1e3,
+                           "entry": "int8_linear_fused_host (pinned host bf16 in, pinned host bf16 out)"}
+
+            # ---- context on the same box: library bf16 matmul and library int8 matmul on the same shapes
+            ctx = []
+            for L in sets[0]:
+                spec = L["spec"]
+                if spec.M <= 16:
+                    continue
+                Wb = torch.randn(spec.N, spec.K, device=dev, dtype=torch.bfloat16)
+                tb = statistics.mean(cuda_timer(torch, lambda: torch.matmul(L["A"], Wb.t()), 10, 3))
+                s_off, q_off = w8.int8_linear_workspace_offsets(spec.M, spec.K)
+                qa = L["ws"][q_off:q_off + spec.M * spec.K].view(torch.int8).view(spec.M, spec.K)
+                ti = statistics.mean(cuda_timer(torch, lambda: torch._int_mm(qa, L["qw"].t()), 10, 3))
+                ctx.append({"name": spec.name, "torch_bf16_matmul_tflops": spec.ops / tb / 1e12,
+                            "torch_int_mm_tops_no_dequant": spec.ops / ti / 1e12})
+                del Wb
+            line["context"] = ctx
+
+            # ---- the oracle on the host cores, bounded sample (only at one GPU)
+            if world == 1:
+                v, sec_o, cores, sample = time_oracle(specs, 1, 0, target_gmac=60.0)
+                line["cpu_baseline"] = {"value": v, "unit": "TOPS", "cores": cores, "kind": "oracle", "sample": sample,
+                                        "seconds": sec_o}
+        print(json.dumps(line), flush=True)
+    wdist.barrier(dev)
+
+
+if __name__ == "__main__":
+    main()

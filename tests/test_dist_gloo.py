@@ -1,0 +1,71 @@
+"""World-size-2 CPU (gloo) test of the benchmark's multi-rank plumbing: row sharding covers the tokens
+exactly once, and whole-job throughput is all ranks' units over the slowest rank's time."""
+import os
+import socket
+import subprocess
+import sys
+import textwrap
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+WORKER = textwrap.dedent("""
+    import json, os, sys
+    sys.path.insert(0, %r)
+    import numpy as np
+    import oracle
+    from paper_2606_14598_b200 import dist as wdist
+    from paper_2606_14598_b200 import inputs as synth
+    rank, local_rank, world = wdist.init("gloo")
+    spec = synth.LinearSpec("gloo", 50, 64, 24)
+    lo, hi = wdist.shard_rows(spec.M, rank, world, multiple=8)
+    # each rank runs the (row-local) path on its own rows; weights are replicated
+    t = synth.make_linear(spec)
+    qw, s_ch = oracle.quantize_weight_per_channel(t["W"].numpy())
+    A = np.ascontiguousarray(synth.bf16_bits(t["A"])[lo:hi])
+    part = oracle.linear_fused_bf16(A, qw, s_ch, t["bias"].numpy())["out"]
+    full = oracle.linear_fused_bf16(synth.bf16_bits(t["A"]), qw, s_ch, t["bias"].numpy())["out"]
+    same = bool((part == full[lo:hi]).all())
+    wdist.barrier()
+    value, tmax = wdist.aggregate_throughput(float(hi - lo), 1.0 + rank)
+    rows_total = wdist.sum_over_ranks(float(hi - lo))
+    print(json.dumps({"rank": rank, "lo": lo, "hi": hi, "same": same, "value": value, "tmax": tmax, "rows": rows_total}))
+""") % ROOT
+
+
+def free_port():
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    p = s.getsockname()[1]
+    s.close()
+    return p
+
+
+def test_two_ranks_gloo():
+    import json
+    port = str(free_port())
+    procs = []
+    for r in range(2):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE="2", MASTER_ADDR="127.0.0.1", MASTER_PORT=port,
+                   OMP_NUM_THREADS="2")
+        procs.append(subprocess.Popen([sys.executable, "-c", WORKER], env=env, stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True))
+    outs = []
+    for p in procs:
+        o, e = p.communicate(timeout=180)
+        assert p.returncode == 0, e[-2000:]
+        outs.append(json.loads(o.strip().splitlines()[-1]))
+    outs.sort(key=lambda d: d["rank"])
+    assert outs[0]["lo"] == 0 and outs[0]["hi"] == outs[1]["lo"] and outs[1]["hi"] == 50
+    assert all(d["same"] for d in outs)                      # sharding over tokens changes no bits
+    assert all(d["rows"] == 50.0 and d["tmax"] == 2.0 and d["value"] == 25.0 for d in outs)
+
+
+def test_shard_rows_partition():
+    from paper_2606_14598_b200.dist import shard_rows
+    for M in (1, 2, 50, 4608, 9216, 4609):
+        for world in (1, 2, 3, 8):
+            for mult in (1, 128):
+                spans = [shard_rows(M, r, world, mult) for r in range(world)]
+                assert spans[0][0] == 0 and spans[-1][1] == M
+                assert all(a[1] == b[0] for a, b in zip(spans, spans[1:]))
+                sizes = [hi - lo for lo, hi in spans]
+                assert max(sizes) - min(sizes) <= 2 * mult - 1
