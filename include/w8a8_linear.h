@@ -83,9 +83,11 @@ int int8_quantize_act_per_token(const void* A_bf16, int64_t M, int64_t K, int64_
  * Bytes of caller-provided device workspace int8_linear_fused needs for this
  * problem (0 on invalid sizes). Layout, from the workspace base (which must be
  * 256-byte aligned): a 256-byte status block; then, for bf16 activations only,
- * s_tok as fp32 [M] (padded to 256 bytes) and qa as int8 [M,K] dense. After a
- * bf16 call the caller may read qa and s_tok back from there
- * (int8_linear_workspace_offsets gives the byte offsets).
+ * one 64-bit progress flag per row (padded to 256 bytes; the quantizer
+ * publishes finished rows there and the GEMM follows them block by block),
+ * s_tok as fp32 [M] (padded to 256 bytes) and qa as int8 [M,K] dense. The
+ * workspace needs no initialisation. After a bf16 call the caller may read qa
+ * and s_tok back from there (int8_linear_workspace_offsets gives the offsets).
  */
 size_t int8_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int a_dtype);
 

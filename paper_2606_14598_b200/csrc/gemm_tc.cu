@@ -3,7 +3,14 @@
 //   acc[m,n] = sum_k qa[m,k] * qw[n,k]        tcgen05.mma.kind::i8, int32 in TMEM
 //   out[m,n] = bf16(((float(acc) * s_tok[m]) * s_ch[n]) + bias[n])
 //
-// One persistent CTA per SM walks output tiles of 128 x BN. Warp roles:
+// One persistent CTA per SM. With CG = 1 every CTA walks output tiles of 128 x BN on its own. With
+// CG = 2 the two CTAs of a cluster form a pair (tcgen05 cta_group::2) that walks tiles of 256 x BN:
+// each CTA loads its own 128 rows of A and its own half (BN/2 rows) of the W tile, the leader CTA
+// issues one MMA for both, and each CTA ends up with its 128 x BN half of the accumulator in its own
+// TMEM. A pair moves half as many W bytes per SM through shared memory as two independent CTAs, which
+// is what the shared-memory bandwidth needs at the int8 rate. No multicast is used anywhere: the
+// leader signals the peer's barriers with a second, plain tcgen05.commit / mbarrier.arrive.
+// Warp roles:
 //   warp 0    TMA producer: loads the 128 x 128-byte A tile and the BN x 128-byte
 //             W tile of each k-block into a ring of shared-memory stages
 //             (128-byte swizzle, K-major: both operands are row-major over K)
@@ -38,12 +45,13 @@ constexpr int NUM_THREADS = 192;
 constexpr int EPI_THREADS = 128;
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;   // 2 s
 
-enum Where { W_PRODUCER_EMPTY = 1, W_MMA_FULL = 2, W_MMA_TMEM_EMPTY = 3, W_EPI_TMEM_FULL = 4, W_DRAIN = 5 };
+enum Where { W_PRODUCER_EMPTY = 1, W_MMA_FULL = 2, W_MMA_TMEM_EMPTY = 3, W_EPI_TMEM_FULL = 4, W_DRAIN = 5, W_QUANT_FLAG = 6 };
 
-template <int BN, int STAGES>
+template <int CG, int BN, int STAGES>
 struct SmemLayout {
     static constexpr int A_BYTES = BM * BK;
-    static constexpr int B_BYTES = BN * BK;
+    static constexpr int B_ROWS = BN / CG;                          // W rows this CTA loads per tile
+    static constexpr int B_BYTES = B_ROWS * BK;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     static constexpr int STAGING_BYTES_PER_WARP = 32 * 128;        // 32 rows x 64 bf16
     static constexpr int OFF_STAGING = STAGES * STAGE_BYTES;
@@ -62,23 +70,28 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-template <int BN, int STAGES, bool RAW_I32>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+// At most 128 registers per thread: the register file then has room for a quantizer CTA (512 threads x 64
+// registers) next to this one, which is what lets the two kernels share an SM.
+template <int CG, int BN, int STAGES, bool RAW_I32>
+__global__ void __maxnreg__(128)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                const __grid_constant__ CUtensorMap tm_out,
                const float* __restrict__ s_tok, const float* __restrict__ s_ch, const float* __restrict__ bias,
-               int32_t* __restrict__ raw_out, int M, int N, int K, int* status, int after_quantizer) {
-    using L = SmemLayout<BN, STAGES>;
+               int32_t* __restrict__ raw_out, int M, int N, int K, int* status, int after_quantizer,
+               const unsigned long long* __restrict__ flags, unsigned long long epoch, int n_fastest) {
+    using L = SmemLayout<CG, BN, STAGES>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = CG == 2 ? cluster_ctarank() : 0u;     // position in the CTA pair; 0 leads
+    const bool leader = rank == 0;
     const uint32_t bars = base + L::OFF_BARS;
-    auto full_bar = [&](int s) { return bars + 8u * s; };
-    auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
-    auto tfull_bar = [&](int b) { return bars + 8u * (2 * STAGES + b); };
-    auto tempty_bar = [&](int b) { return bars + 8u * (2 * STAGES + 2 + b); };
+    auto full_bar = [&](int s) { return bars + 8u * s; };                      // used in the leader
+    auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };          // one per CTA
+    auto tfull_bar = [&](int b) { return bars + 8u * (2 * STAGES + b); };      // one per CTA
+    auto tempty_bar = [&](int b) { return bars + 8u * (2 * STAGES + 2 + b); }; // used in the leader
     volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(base_ptr + L::OFF_TMEM);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::OFF_ABORT);
     const WaitCtl ctl{abort_flag, status, WAIT_LIMIT_NS};
@@ -87,7 +100,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
+        for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4 * CG); }
         *abort_flag = 0;
         fence_mbar_init();
         prefetch_tensormap(&tm_a);
@@ -95,59 +108,91 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         if (!RAW_I32) prefetch_tensormap(&tm_out);
     }
     if (warp == 1) {
-        tmem_alloc(base + L::OFF_TMEM, TMEM_COLS);
-        tmem_relinquish();
+        if (CG == 2) { tmem_alloc_pair(base + L::OFF_TMEM, TMEM_COLS); tmem_relinquish_pair(); }
+        else { tmem_alloc(base + L::OFF_TMEM, TMEM_COLS); tmem_relinquish(); }
     }
     tc_fence_before();
     __syncthreads();
+    if (CG == 2) cluster_sync_all();            // the peer's barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_holder;
 
-    const int num_m = (M + BM - 1) / BM, num_n = (N + BN - 1) / BN;
+    constexpr int TILE_M = BM * CG;
+    const int num_m = (M + TILE_M - 1) / TILE_M, num_n = (N + BN - 1) / BN;
     const int num_tiles = num_m * num_n;
     const int num_kb = (K + BK - 1) / BK;
+    const int first_tile = blockIdx.x / CG, tile_step = gridDim.x / CG;
+    // tile order: along M first (neighbouring CTAs share a W tile), or along N first (the first tiles
+    // need only the first rows of A, which lets the kernel start while the quantizer is still running)
+    auto tile_m = [&](int t) { return n_fastest ? t / num_n : t % num_m; };
+    auto tile_n = [&](int t) { return n_fastest ? t % num_n : t / num_m; };
+    // row r is quantized once flags[r] carries this call's epoch; a warp checks the BM rows of a block
+    auto rows_ready = [&](int m0, int where) {
+        bool ok = true;
+        for (int r = m0 + lane; r < min(m0 + BM, M) && ok; r += 32)
+            ok = flag_wait(flags + r, epoch, ctl, where, kStatusTimeout);
+        return __all_sync(0xffffffffu, ok) != 0;
+    };
 
     if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            if (after_quantizer) grid_dep_wait();      // qa / s_tok come from the kernel before this one
-            int stage = 0;
-            uint32_t phase = 0;
-            int issued = 0;
-            bool ok = true;
-            for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
-                const int m0 = (t % num_m) * BM, n0 = (t / num_m) * BN;
+        // ------------------------------------------------------------ TMA producer (both CTAs of a pair)
+        if (after_quantizer && flags == nullptr && lane == 0) grid_dep_wait();   // qa comes from the kernel before this one
+        __syncwarp();
+        int stage = 0;
+        uint32_t phase = 0;
+        int issued = 0;
+        bool ok = true;
+        int ready_m0 = -1;
+        for (int t = first_tile; t < num_tiles && ok; t += tile_step) {
+            const int m0 = tile_m(t) * TILE_M + rank * BM;
+            const int n0 = tile_n(t) * BN + rank * L::B_ROWS;
+            if (flags != nullptr && m0 != ready_m0 && m0 < M) {      // all lanes poll, one flag per row
+                if (!rows_ready(m0, W_QUANT_FLAG)) { ok = false; break; }
+                ready_m0 = m0;
+            }
+            if (lane == 0) {
+                const uint64_t keep = l2_policy_evict_last();        // operands are re-read by other tiles: keep them in L2
+                if (flags != nullptr) fence_proxy_async_all();       // the TMA reads below come after the acquire
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, ctl, W_PRODUCER_EMPTY, kStatusTimeout)) { ok = false; break; }
-                    mbar_arrive_expect_tx(full_bar(stage), L::STAGE_BYTES);
                     const uint32_t sa = base + stage * L::STAGE_BYTES;
-                    tma_load_2d(sa, &tm_a, full_bar(stage), kb * BK, m0);
-                    tma_load_2d(sa + L::A_BYTES, &tm_b, full_bar(stage), kb * BK, n0);
+                    if (CG == 2) {
+                        // the leader's barrier counts the bytes of both CTAs
+                        if (leader) mbar_arrive_expect_tx(full_bar(stage), 2 * L::STAGE_BYTES);
+                        const uint32_t fb = mapa_shared(full_bar(stage), 0);
+                        tma_load_2d_pair_hint(sa, &tm_a, fb, kb * BK, m0, keep);
+                        tma_load_2d_pair_hint(sa + L::A_BYTES, &tm_b, fb, kb * BK, n0, keep);
+                    } else {
+                        mbar_arrive_expect_tx(full_bar(stage), L::STAGE_BYTES);
+                        tma_load_2d_hint(sa, &tm_a, full_bar(stage), kb * BK, m0, keep);
+                        tma_load_2d_hint(sa + L::A_BYTES, &tm_b, full_bar(stage), kb * BK, n0, keep);
+                    }
                     ++issued;
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
-            if (!ok) {
-                // let copies that are still in flight land before the CTA goes away
-                int s = stage;
-                uint32_t ph = phase;
-                for (int i = 0; i < STAGES && i < issued; ++i) {
-                    if (s == 0) { s = STAGES; ph ^= 1u; }
-                    --s;
-                    const uint64_t t0 = globaltimer_ns();
-                    while (!mbar_try_wait(full_bar(s), ph) && globaltimer_ns() - t0 < 10000000ull) {}
-                }
+            ok = __all_sync(0xffffffffu, ok) != 0;
+        }
+        if (!ok && lane == 0 && (CG == 1 || leader)) {
+            // let copies that are still in flight land before the CTA goes away
+            int s = stage;
+            uint32_t ph = phase;
+            for (int i = 0; i < STAGES && i < issued; ++i) {
+                if (s == 0) { s = STAGES; ph ^= 1u; }
+                --s;
+                const uint64_t t0 = globaltimer_ns();
+                while (!mbar_try_wait(full_bar(s), ph) && globaltimer_ns() - t0 < 10000000ull) {}
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc = make_i8_idesc(BM, BN);
+        // ------------------------------------------------------------ MMA issuer (leader CTA only)
+        if (lane == 0 && leader) {
+            constexpr uint32_t idesc = make_i8_idesc(TILE_M, BN);
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
             int it = 0;
-            for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++it) {
+            for (int t = first_tile; t < num_tiles && ok; t += tile_step, ++it) {
                 const int buf = it & 1;
                 if (!mbar_wait(tempty_bar(buf), ((it >> 1) & 1) ^ 1u, ctl, W_MMA_TMEM_EMPTY, kStatusTimeout)) { ok = false; break; }
                 tc_fence_after();
@@ -161,13 +206,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     const int ksteps = min(BK, K - kb * BK + MMA_K - 1) / MMA_K;   // skip all-zero tail steps
 #pragma unroll
                     for (int k = 0; k < BK / MMA_K; ++k) {
-                        if (k < ksteps)   // advancing K by 32 bytes inside the swizzled row: +2 in 16-byte units
-                            mma_i8_ss(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                        if (k < ksteps) {   // advancing K by 32 bytes inside the swizzled row: +2 in 16-byte units
+                            if (CG == 2) mma_i8_ss_pair(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                            else mma_i8_ss(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                        }
                     }
-                    tc_commit(empty_bar(stage));          // stage is free once these MMAs have read it
+                    // the stage is free (in both CTAs) once these MMAs have read it
+                    if (CG == 2) { tc_commit_pair(empty_bar(stage)); tc_commit_pair(mapa_shared(empty_bar(stage), 1)); }
+                    else tc_commit(empty_bar(stage));
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
-                if (ok) tc_commit(tfull_bar(buf));        // accumulator complete
+                if (ok) {                                  // accumulator complete (in both CTAs)
+                    if (CG == 2) { tc_commit_pair(tfull_bar(buf)); tc_commit_pair(mapa_shared(tfull_bar(buf), 1)); }
+                    else tc_commit(tfull_bar(buf));
+                }
             }
         }
     } else {
@@ -179,12 +231,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         const uint32_t staging = base + L::OFF_STAGING + (warp - 2) * L::STAGING_BYTES_PER_WARP;
         uint8_t* staging_ptr = base_ptr + L::OFF_STAGING + (warp - 2) * L::STAGING_BYTES_PER_WARP;
         const bool has_bias = bias != nullptr;
-        if (after_quantizer) grid_dep_wait();          // s_tok comes from the kernel before this one
+        const uint64_t stream_out = l2_policy_evict_first();        // the output is written once and not read here
+        if (after_quantizer && flags == nullptr) grid_dep_wait();   // s_tok comes from the kernel before this one
         bool ok = true;
         int it = 0;
-        for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
+        int ready_m0 = -1;
+        for (int t = first_tile; t < num_tiles; t += tile_step, ++it) {
             const int buf = it & 1;
-            const int m0 = (t % num_m) * BM, n0 = (t / num_m) * BN;
+            const int m0 = tile_m(t) * TILE_M + rank * BM, n0 = tile_n(t) * BN;
+            if (flags != nullptr && ok && m0 != ready_m0) {             // s_tok of this thread's row is published
+                const int r = m0 + lg * 32 + lane;
+                const bool mine = r >= M || flag_wait(flags + r, epoch, ctl, W_QUANT_FLAG, kStatusTimeout);
+                if (!__all_sync(0xffffffffu, mine)) ok = false;
+                ready_m0 = m0;
+            }
             if (!RAW_I32) {
                 asm volatile("bar.sync 1, 128;" ::: "memory");     // previous tile's readers are done
                 for (int j = ep_tid; j < BN; j += EPI_THREADS) {
@@ -202,59 +262,61 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             tc_fence_after();
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(lg * 32) << 16) + buf * BN;
 #pragma unroll 1
-            for (int c = 0; c < BN / 64; ++c) {
-                uint32_t v0[32], v1[32];
-                tmem_ld_32x32b_x32(t_row + c * 64, v0);
-                tmem_ld_32x32b_x32(t_row + c * 64 + 32, v1);
-                tmem_wait_ld();
-                if (c == BN / 64 - 1) {                // accumulator fully read: hand the buffer back
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(tempty_bar(buf));
+            for (int c = 0; c < BN / 64; ++c) {        // one 32 x 64 output box per iteration
+#pragma unroll 1
+                for (int h = 0; h < 2; ++h) {          // in two halves of 32 columns (keeps registers low)
+                    const int col = c * 64 + h * 32;
+                    uint32_t v[32];
+                    tmem_ld_32x32b_x32(t_row + col, v);
+                    tmem_wait_ld();
+                    if (c == BN / 64 - 1 && h == 1) {  // accumulator fully read: hand the buffer back
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) {
+                            if (CG == 2) mbar_arrive_cluster(mapa_shared(tempty_bar(buf), 0));
+                            else mbar_arrive(tempty_bar(buf));
+                        }
+                    }
+                    if (RAW_I32) {
+                        if (row < M) {
+                            int32_t* dst = raw_out + static_cast<int64_t>(row) * N + n0 + col;
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (n0 + col + j < N) dst[j] = static_cast<int32_t>(v[j]);
+                        }
+                    } else {
+                        uint32_t packed[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const float2 sc = *reinterpret_cast<const float2*>(sm_sch + col + 2 * j);
+                            float a0 = __fmul_rn(__fmul_rn(__int2float_rn(static_cast<int>(v[2 * j])), st), sc.x);
+                            float a1 = __fmul_rn(__fmul_rn(__int2float_rn(static_cast<int>(v[2 * j + 1])), st), sc.y);
+                            if (has_bias) {
+                                const float2 bi = *reinterpret_cast<const float2*>(sm_bias + col + 2 * j);
+                                a0 = __fadd_rn(a0, bi.x);
+                                a1 = __fadd_rn(a1, bi.y);
+                            }
+                            packed[j] = pack_bf16x2(a0, a1);
+                        }
+                        if (h == 0) {
+                            // the previous TMA store must have finished reading the staging buffer
+                            if (lane == 0) bulk_wait_group_read<0>();
+                            __syncwarp();
+                        }
+                        // row `lane` of the 32 x 128-byte box; 16-byte chunk i lives at chunk (i ^ (row & 7))
+                        uint8_t* srow = staging_ptr + lane * 128;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            uint4 q = make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
+                            *reinterpret_cast<uint4*>(srow + (((h * 4 + i) ^ (lane & 7)) << 4)) = q;
+                        }
+                    }
                 }
-                if (RAW_I32) {
-                    if (row < M) {
-                        int32_t* dst = raw_out + static_cast<int64_t>(row) * N + n0 + c * 64;
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            if (n0 + c * 64 + j < N) dst[j] = static_cast<int32_t>(v0[j]);
-                            if (n0 + c * 64 + 32 + j < N) dst[32 + j] = static_cast<int32_t>(v1[j]);
-                        }
-                    }
-                } else {
-                    uint32_t packed[32];
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        // columns c*64 + 2j, +1 (from v0) and c*64 + 32 + 2j, +1 (from v1)
-                        const float2 sc0 = *reinterpret_cast<const float2*>(sm_sch + c * 64 + 2 * j);
-                        const float2 sc1 = *reinterpret_cast<const float2*>(sm_sch + c * 64 + 32 + 2 * j);
-                        float a0 = __fmul_rn(__fmul_rn(__int2float_rn(static_cast<int>(v0[2 * j])), st), sc0.x);
-                        float a1 = __fmul_rn(__fmul_rn(__int2float_rn(static_cast<int>(v0[2 * j + 1])), st), sc0.y);
-                        float b0 = __fmul_rn(__fmul_rn(__int2float_rn(static_cast<int>(v1[2 * j])), st), sc1.x);
-                        float b1 = __fmul_rn(__fmul_rn(__int2float_rn(static_cast<int>(v1[2 * j + 1])), st), sc1.y);
-                        if (has_bias) {
-                            const float2 bi0 = *reinterpret_cast<const float2*>(sm_bias + c * 64 + 2 * j);
-                            const float2 bi1 = *reinterpret_cast<const float2*>(sm_bias + c * 64 + 32 + 2 * j);
-                            a0 = __fadd_rn(a0, bi0.x); a1 = __fadd_rn(a1, bi0.y);
-                            b0 = __fadd_rn(b0, bi1.x); b1 = __fadd_rn(b1, bi1.y);
-                        }
-                        packed[j] = pack_bf16x2(a0, a1);
-                        packed[16 + j] = pack_bf16x2(b0, b1);
-                    }
-                    // the previous TMA store must have finished reading the staging buffer
-                    if (lane == 0) bulk_wait_group_read<0>();
-                    __syncwarp();
-                    // row `lane` of the 32 x 128-byte box; 16-byte chunk i lives at chunk (i ^ (row & 7))
-                    uint8_t* srow = staging_ptr + lane * 128;
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        uint4 q = make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
-                        *reinterpret_cast<uint4*>(srow + ((i ^ (lane & 7)) << 4)) = q;
-                    }
+                if (!RAW_I32) {
                     fence_proxy_async_smem();
                     __syncwarp();
                     if (lane == 0) {
-                        tma_store_2d(&tm_out, staging, n0 + c * 64, m0 + lg * 32);
+                        tma_store_2d_hint(&tm_out, staging, n0 + c * 64, m0 + lg * 32, stream_out);
                         bulk_commit_group();
                     }
                 }
@@ -263,10 +325,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         if (!RAW_I32 && lane == 0) bulk_wait_group<0>();
     }
 
+    // this grid may only count as complete once the quantizer grid before it has completed
+    if (after_quantizer && flags != nullptr && threadIdx.x == 0) grid_dep_wait();
     tc_fence_before();
     __syncthreads();
+    if (CG == 2) cluster_sync_all();            // nobody leaves while the peer may still signal its barriers
     tc_fence_after();
-    if (warp == 1) tmem_dealloc(tmem_base, TMEM_COLS);
+    if (warp == 1) {
+        if (CG == 2) tmem_dealloc_pair(tmem_base, TMEM_COLS);
+        else tmem_dealloc(tmem_base, TMEM_COLS);
+    }
 }
 
 // ---------------------------------------------------------------------------- host side
@@ -302,11 +370,13 @@ bool encode_2d(CUtensorMap* tm, CUtensorMapDataType dt, const void* ptr, uint64_
 
 struct TcConfig {
     const char* name;
-    int bn, stages;
+    int cg, bn, stages;
 };
 constexpr TcConfig kConfigs[] = {
-    {"tc 128x256 4 stages", 256, 4},
-    {"tc 128x128 6 stages", 128, 6},
+    {"tc 128x256 per CTA, 4 stages", 1, 256, 4},
+    {"tc 128x128 per CTA, 6 stages", 1, 128, 6},
+    {"tc 256x256 per CTA pair, 6 stages", 2, 256, 6},
+    {"tc 256x128 per CTA pair, 8 stages", 2, 128, 8},
 };
 constexpr int kNumConfigs = sizeof(kConfigs) / sizeof(kConfigs[0]);
 
@@ -320,11 +390,11 @@ int sm_count() {
     return n;
 }
 
-template <int BN, int STAGES, bool RAW>
+template <int CG, int BN, int STAGES, bool RAW>
 int launch_cfg(const GemmArgs& a, cudaStream_t st) {
-    using L = SmemLayout<BN, STAGES>;
+    using L = SmemLayout<CG, BN, STAGES>;
     static_assert(L::DYN_BYTES <= 232448, "shared memory budget");
-    auto kern = gemm_tc_kernel<BN, STAGES, RAW>;
+    auto kern = gemm_tc_kernel<CG, BN, STAGES, RAW>;
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [&] { attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES); });
@@ -332,34 +402,48 @@ int launch_cfg(const GemmArgs& a, cudaStream_t st) {
 
     CUtensorMap tm_a, tm_b, tm_out;
     if (!encode_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, a.qa, a.M, a.K, a.lda_q, BM, BK)) return 6;
-    if (!encode_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, a.qw, a.N, a.K, a.K, BN, BK)) return 6;
+    if (!encode_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, a.qw, a.N, a.K, a.K, L::B_ROWS, BK)) return 6;
     if (RAW) {
         tm_out = tm_a;   // unused
     } else {
         if (!encode_2d(&tm_out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, a.out, a.M, a.N, a.ldo * 2, 32, 64)) return 6;
     }
-    const int num_tiles = ((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN);
+    const int num_tiles = ((a.M + BM * CG - 1) / (BM * CG)) * ((a.N + BN - 1) / BN);
+    const int max_groups = sm_count() / CG;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(num_tiles < sm_count() ? num_tiles : sm_count());
+    cfg.gridDim = dim3(CG * (num_tiles < max_groups ? num_tiles : max_groups));
     cfg.blockDim = dim3(NUM_THREADS);
     cfg.dynamicSmemBytes = L::DYN_BYTES;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute attr[2];
+    int na = 0;
+    if (CG == 2) {
+        attr[na].id = cudaLaunchAttributeClusterDimension;
+        attr[na].val.clusterDim.x = 2;
+        attr[na].val.clusterDim.y = 1;
+        attr[na].val.clusterDim.z = 1;
+        ++na;
+    }
+    if (a.after_quantizer) {
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = a.after_quantizer ? 1 : 0;
+    cfg.numAttrs = na;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tm_a, tm_b, tm_out, a.s_tok, a.s_ch, a.bias,
                                        RAW ? static_cast<int32_t*>(a.out) : nullptr, a.M, a.N, a.K, a.status,
-                                       a.after_quantizer ? 1 : 0);
+                                       a.after_quantizer ? 1 : 0, a.flags, a.epoch, a.flags != nullptr ? 1 : 0);
     return e == cudaSuccess ? 0 : 6;
 }
 
 template <bool RAW>
 int launch_by_id(int id, const GemmArgs& a, cudaStream_t st) {
     switch (id) {
-        case 0: return launch_cfg<256, 4, RAW>(a, st);
-        case 1: return launch_cfg<128, 6, RAW>(a, st);
+        case 0: return launch_cfg<1, 256, 4, RAW>(a, st);
+        case 1: return launch_cfg<1, 128, 6, RAW>(a, st);
+        case 2: return launch_cfg<2, 256, 6, RAW>(a, st);
+        case 3: return launch_cfg<2, 128, 8, RAW>(a, st);
         default: return 1;
     }
 }
@@ -376,6 +460,16 @@ int pick_config(int M, int N, int K) {
 
 int tc_num_configs() { return kNumConfigs; }
 const char* tc_config_name(int id) { return (id >= 0 && id < kNumConfigs) ? kConfigs[id].name : nullptr; }
+
+int tc_first_wave_rows(int M, int N, int K, int forced) {
+    const int id = (forced >= 0 && forced < kNumConfigs) ? forced : pick_config(M, N, K);
+    const int tile_m = BM * kConfigs[id].cg, bn = kConfigs[id].bn;
+    const int num_n = (N + bn - 1) / bn;
+    const int groups = sm_count() / kConfigs[id].cg;             // tiles in flight at once
+    const int m_blocks = (groups + num_n - 1) / num_n;          // N-fastest order: rows of that many row blocks
+    const long rows = static_cast<long>(m_blocks) * tile_m;
+    return rows < M ? static_cast<int>(rows) : M;
+}
 
 int launch_gemm_tc(const GemmArgs& a, int forced, cudaStream_t st) {
     const int id = (forced >= 0 && forced < kNumConfigs) ? forced : pick_config(a.M, a.N, a.K);

@@ -79,6 +79,35 @@ def test_act_quantizer_bit_exact(M, K):
     assert np.array_equal(qa.cpu().numpy(), qa_ref)
 
 
+def test_act_quantizer_every_bf16_value_against_many_scales():
+    """Exhaustive in x: every finite bf16 value not above the row's absmax, for 320 different absmax
+    values (random ones, all-ones and all-zeros mantissas, tiny and huge exponents). bf16 inputs make
+    exact rounding ties common, so this is where a quotient that is off by one ulp would show."""
+    rng = np.random.default_rng(2024)
+    pats = np.arange(65536, dtype=np.uint32)
+    finite = (pats & 0x7F80) != 0x7F80
+    vals = np.where(finite, pats, 0).astype(np.uint16)                      # NaN / Inf patterns -> +0
+    mags = (vals & 0x7FFF).astype(np.int64)
+    amax_bits = np.concatenate([
+        rng.integers(0x3000, 0x4F00, 256),                                   # ordinary magnitudes
+        np.array([0x3F80, 0x3FFF, 0x407F, 0x42FE, 0x4000, 0x3F7F, 0x437F, 0x3E00]),   # 1, all-ones mantissas, 127, 255 ...
+        rng.integers(0x0080, 0x0800, 24), rng.integers(0x7000, 0x7F7F, 32)]).astype(np.int64)   # tiny / huge
+    rows = []
+    for ab in amax_bits:
+        row = np.where(mags <= ab, vals, 0).astype(np.uint16)
+        row = row.reshape(8, 8192).copy()
+        row[:, 0] = ab                                                       # every row carries its absmax
+        rows.append(row)
+    A_bits = np.ascontiguousarray(np.concatenate(rows, axis=0))
+    qa_ref, s_ref = oracle.quantize_act_per_token(A_bits)
+    A = synth.bits_to_bf16(A_bits).to(DEV)
+    qa, s = w8.int8_quantize_act_per_token(A)
+    assert np.array_equal(s.cpu().numpy().view(np.uint32), s_ref.view(np.uint32))
+    got = qa.cpu().numpy()
+    bad = np.argwhere(got != qa_ref)
+    assert bad.size == 0, f"{len(bad)} codes differ, first at {bad[0]}: got {got[tuple(bad[0])]} want {qa_ref[tuple(bad[0])]}"
+
+
 def test_act_quantizer_gelu_rows_and_row_stride():
     spec = synth.LinearSpec("qg", 70, 1024, 8, act="gelu", outlier_frac=0.0)
     A = synth.make_activations(spec)
@@ -304,6 +333,10 @@ def test_benchmark_configs_full_size(spec):
     ridx = torch.from_numpy(rows).to(DEV)
     assert np.array_equal(s_tok[ridx].cpu().numpy(), ref["s_tok"])
     assert np.array_equal(qa[ridx].cpu().numpy(), ref["qa"])
+    # the quantizer is cheap for the oracle too: compare every code and every scale of the whole tensor
+    qa_full, s_full = oracle.quantize_act_per_token(synth.bf16_bits(t["A"]))
+    assert np.array_equal(s_tok.cpu().numpy(), s_full)
+    assert np.array_equal(qa.cpu().numpy(), qa_full)
     assert_bf16_close(synth.bf16_bits(out[ridx].cpu()), ref["out"])
     # raw accumulators: sampled rows vs the oracle, everything vs the library integer matmul
     acc = w8.int8_gemm_i32_debug(qa, qw)
