@@ -134,6 +134,40 @@ int int8_linear_fused_host(const void* A_host, void* d_A,
                            void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Allocation-free variant of the fused linear on bf16 activations. (The paper has no counterpart: it is
+ * an interface convenience of this library.)
+ *
+ * For callers that cannot provide a workspace because they cannot allocate one: a server whose own arena
+ * already owns all device memory, a latency-critical loop where cudaMalloc's implicit synchronisation is
+ * not acceptable, a plug-in that only ever receives its input and output buffers. The scratch that
+ * int8_linear_fused takes from the caller (status word, per-row progress flags, s_tok, qa) is a fixed
+ * array of W8A8_STATIC_WORKSPACE_BYTES inside the library's device image; every GPU that loads the library
+ * holds that much memory until the process exits. The call itself allocates nothing (no cudaMalloc,
+ * cudaFree or allocating library routine).
+ *
+ *   Arguments as for int8_linear_fused with a_dtype == W8A8_ACT_BF16 (device pointers, caller-owned).
+ *   sync_and_check  0: enqueue and return. Non-zero: additionally synchronize `stream` and return
+ *                   W8A8_ERR_TIMEOUT if a bounded device-side wait gave up (as int8_check_status does).
+ *
+ * Limits and rules:
+ *   - Problems whose scratch, int8_linear_workspace_bytes(M, N, K, W8A8_ACT_BF16), exceeds
+ *     W8A8_STATIC_WORKSPACE_BYTES are refused with W8A8_ERR_WORKSPACE before anything is enqueued
+ *     (roughly M * (K + 12) <= 16 MiB: e.g. M = 4608 tokens at K = 3072, not at K = 12288).
+ *   - The first call on each device looks up the array's device address (a one-time set-up step under a
+ *     mutex). Make that first call outside any stream capture.
+ *   - All calls on a device share the one array. Calls on the same stream run one after the other and are
+ *     safe; calls that may overlap on the GPU (different streams, different host threads) race on it and
+ *     must be serialized by the caller, or use int8_linear_fused with separate workspaces.
+ *   - The array keeps whatever the last call left in it. Nothing needs clearing: each call resets the
+ *     status word and uses a fresh progress-flag value.
+ */
+#define W8A8_STATIC_WORKSPACE_BYTES (16u * 1024u * 1024u)
+int int8_linear_fused_static(const void* A_bf16, int64_t lda,
+                             const int8_t* qw, const float* s_ch, const float* bias,
+                             void* out_bf16, int64_t ldo, int64_t M, int64_t N, int64_t K,
+                             int sync_and_check, void* stream);
+
+/*
  * Test-only export of the raw accumulators of the tensor-core path (the int32
  * values the fused epilogue consumes): acc[m,n] = sum_k qa[m,k] * qw[n,k].
  *   qa in int8 [M,K] dense; qw in int8 [N,K] dense; acc out int32 [M,N] dense (N % 4 == 0);

@@ -25,7 +25,7 @@ EXPORTS = (
     "int8_quantize_weight_per_channel", "int8_quantize_act_per_token", "int8_linear_workspace_bytes",
     "int8_linear_workspace_offsets", "int8_linear_fused", "int8_linear_fused_host", "int8_gemm_i32_debug",
     "int8_check_status", "int8_linear_force_config", "int8_linear_num_configs", "int8_linear_config_name",
-    "int8_status_string",
+    "int8_status_string", "int8_linear_fused_static",
 )
 
 if not os.path.exists(LIB_PATH):
@@ -48,6 +48,8 @@ _lib.int8_linear_fused.argtypes = [_vp, _int, _i64, _vp, _vp, _vp, _vp, _vp, _i6
 _lib.int8_linear_fused.restype = _int
 _lib.int8_linear_fused_host.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp, _sz, _vp]
 _lib.int8_linear_fused_host.restype = _int
+_lib.int8_linear_fused_static.argtypes = [_vp, _i64, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i64, _int, _vp]
+_lib.int8_linear_fused_static.restype = _int
 _lib.int8_gemm_i32_debug.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64, _vp, _sz, _vp]
 _lib.int8_gemm_i32_debug.restype = _int
 _lib.int8_check_status.argtypes = [_vp, _vp]
@@ -198,6 +200,32 @@ def int8_linear_fused_host(A_host: torch.Tensor, d_A: torch.Tensor, qw: torch.Te
                                        _ptr(out_host), M, N, K, _ptr(workspace), workspace.numel(), _stream(d_A)),
            "int8_linear_fused_host")
     return out_host
+
+
+STATIC_WORKSPACE_BYTES = 16 * 1024 * 1024
+
+
+def int8_linear_fused_static(A: torch.Tensor, qw: torch.Tensor, s_ch: torch.Tensor, bias: torch.Tensor | None = None,
+                             out: torch.Tensor | None = None, sync_and_check: bool = False) -> torch.Tensor:
+    """Fused linear on bf16 activations whose scratch is the library's built-in device array: no workspace
+    argument and no allocation inside the call. For callers that cannot allocate (see the header). Refuses
+    problems whose scratch exceeds STATIC_WORKSPACE_BYTES; calls that overlap on the GPU share the array and race."""
+    _need(A, torch.bfloat16, "A", 2)
+    _need(qw, torch.int8, "qw", 2)
+    _need(s_ch, torch.float32, "s_ch", 1)
+    M, K = A.shape
+    N = qw.shape[0]
+    if qw.shape[1] != K or s_ch.shape[0] != N or not qw.is_contiguous():
+        raise ValueError("shape mismatch")
+    if bias is not None:
+        _need(bias, torch.float32, "bias", 1)
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=A.device)   # the caller's output, not scratch
+    _need(out, torch.bfloat16, "out", 2)
+    _check(_lib.int8_linear_fused_static(_ptr(A), A.stride(0), _ptr(qw), _ptr(s_ch), _ptr(bias), _ptr(out),
+                                         out.stride(0), M, N, K, 1 if sync_and_check else 0, _stream(A)),
+           "int8_linear_fused_static")
+    return out
 
 
 def int8_gemm_i32_debug(qa: torch.Tensor, qw: torch.Tensor, workspace: torch.Tensor | None = None) -> torch.Tensor:
