@@ -165,8 +165,8 @@ int int8_linear_fused(const void* A, int a_dtype, int64_t lda, const float* s_to
             return W8A8_ERR_CUDA;
         g.qa = qa; g.lda_q = K; g.s_tok = s_tok; g.after_quantizer = true; g.flags = flags; g.epoch = epoch;
     } else {
-        if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return W8A8_ERR_CUDA;
         g.qa = static_cast<const int8_t*>(A); g.lda_q = lda; g.s_tok = s_tok_in; g.after_quantizer = false;
+        g.epoch = next_epoch();
     }
     const int forced = g_forced_config.load();
     if ((forced < 0 && M <= kSkinnyM) || forced == tc_num_configs())
@@ -206,7 +206,7 @@ int int8_gemm_i32_debug(const int8_t* qa, const int8_t* qw, int32_t* acc,
     GemmArgs g{};
     g.qa = qa; g.lda_q = K; g.s_tok = nullptr; g.qw = qw; g.s_ch = nullptr; g.bias = nullptr;
     g.out = acc; g.ldo = N; g.M = static_cast<int>(M); g.N = static_cast<int>(N); g.K = static_cast<int>(K);
-    g.raw_i32 = true; g.status = status; g.after_quantizer = false;
+    g.raw_i32 = true; g.status = status; g.after_quantizer = false; g.epoch = next_epoch();
     const int forced = g_forced_config.load();
     if ((forced < 0 && M <= kSkinnyM) || forced == tc_num_configs())
         return launch_gemm_simt(g, st) == cudaSuccess ? W8A8_OK : W8A8_ERR_CUDA;

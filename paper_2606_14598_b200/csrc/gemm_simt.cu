@@ -25,7 +25,9 @@ template <int MB, int NPW, int WARPS>
 __global__ void __launch_bounds__(WARPS * 32)
 gemm_simt_kernel(const int8_t* __restrict__ qa, int64_t lda_q, const float* __restrict__ s_tok,
                  const int8_t* __restrict__ qw, const float* __restrict__ s_ch, const float* __restrict__ bias,
-                 void* __restrict__ out, int64_t ldo, int M, int N, int K, int raw_i32, int after_quantizer) {
+                 void* __restrict__ out, int64_t ldo, int M, int N, int K, int raw_i32, int after_quantizer, int* status) {
+    // no quantizer ahead of this kernel to clear the status word: do it here (this kernel has no waits that could set it)
+    if (!after_quantizer && status != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *status = 0;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n0 = (blockIdx.x * WARPS + warp) * NPW;
     const int m0 = blockIdx.y * MB;
@@ -102,7 +104,7 @@ cudaError_t launch(const GemmArgs& a, cudaStream_t st) {
     cfg.attrs = attr;
     cfg.numAttrs = a.after_quantizer ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, gemm_simt_kernel<MB, NPW, WARPS>, a.qa, a.lda_q, a.s_tok, a.qw, a.s_ch, a.bias,
-                              a.out, a.ldo, a.M, a.N, a.K, a.raw_i32 ? 1 : 0, a.after_quantizer ? 1 : 0);
+                              a.out, a.ldo, a.M, a.N, a.K, a.raw_i32 ? 1 : 0, a.after_quantizer ? 1 : 0, a.status);
 }
 
 } // namespace

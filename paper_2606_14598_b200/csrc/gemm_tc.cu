@@ -32,8 +32,8 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <cstdlib>
 #include <mutex>
-#include <unordered_map>
 
 namespace w8a8 {
 namespace {
@@ -53,7 +53,10 @@ struct SmemLayout {
     static constexpr int B_ROWS = BN / CG;                          // W rows this CTA loads per tile
     static constexpr int B_BYTES = B_ROWS * BK;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int STAGING_BYTES_PER_WARP = 32 * 128;        // 32 rows x 64 bf16
+    static constexpr int STAGING_BOX_BYTES = 32 * 128;             // one 32-row x 64-column bf16 box
+    // two boxes alternate per epilogue warp where shared memory allows, else one
+    static constexpr int STAGING_BUFS = (STAGES * STAGE_BYTES + 8 * STAGING_BOX_BYTES + 8 * BN + 1280 <= 232448) ? 2 : 1;
+    static constexpr int STAGING_BYTES_PER_WARP = STAGING_BUFS * STAGING_BOX_BYTES;
     static constexpr int OFF_STAGING = STAGES * STAGE_BYTES;
     static constexpr int OFF_SCH = OFF_STAGING + 4 * STAGING_BYTES_PER_WARP;
     static constexpr int OFF_BIAS = OFF_SCH + BN * 4;
@@ -78,7 +81,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                const __grid_constant__ CUtensorMap tm_out,
                const float* __restrict__ s_tok, const float* __restrict__ s_ch, const float* __restrict__ bias,
                int32_t* __restrict__ raw_out, int M, int N, int K, int* status, int after_quantizer,
-               const unsigned long long* __restrict__ flags, unsigned long long epoch, int n_fastest) {
+               const unsigned long long* __restrict__ flags, unsigned long long epoch, int raster_gn) {
     using L = SmemLayout<CG, BN, STAGES>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -98,6 +101,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 
     constexpr uint32_t TMEM_COLS = 2 * BN;      // 512 or 256: a power of two >= 32
 
+    // without a quantizer ahead of it (which clears the status word) the kernel clears it itself; a time-out
+    // can only be recorded seconds later
+    if (!after_quantizer && blockIdx.x == 0 && threadIdx.x == 0) *status = 0;
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4 * CG); }
@@ -122,10 +128,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     const int num_tiles = num_m * num_n;
     const int num_kb = (K + BK - 1) / BK;
     const int first_tile = blockIdx.x / CG, tile_step = gridDim.x / CG;
-    // tile order: along M first (neighbouring CTAs share a W tile), or along N first (the first tiles
-    // need only the first rows of A, which lets the kernel start while the quantizer is still running)
-    auto tile_m = [&](int t) { return n_fastest ? t / num_n : t % num_m; };
-    auto tile_n = [&](int t) { return n_fastest ? t % num_n : t / num_m; };
+    // Tile order: bands of raster_gn tile columns; inside a band the column index runs fastest, then the
+    // row block. raster_gn = 1 walks along M first, raster_gn >= num_n along N first. A wave of concurrent
+    // tiles then covers about (wave / gn) row blocks x gn columns: A and W lines are shared by a balanced
+    // number of CTAs, and (for the from-bf16 entry) the first wave needs only the first row blocks of A.
+    const int gn = raster_gn < 1 ? 1 : (raster_gn > num_n ? num_n : raster_gn);
+    const int band_tiles = num_m * gn;
+    auto tile_n = [&](int t) {
+        const int band = t / band_tiles, r = t - band * band_tiles;
+        const int w = min(gn, num_n - band * gn);               // the last band may be narrower
+        return band * gn + r % w;
+    };
+    auto tile_m = [&](int t) {
+        const int band = t / band_tiles, r = t - band * band_tiles;
+        const int w = min(gn, num_n - band * gn);
+        return r / w;
+    };
     // row r is quantized once flags[r] carries this call's epoch; a warp checks the BM rows of a block
     auto rows_ready = [&](int m0, int where) {
         bool ok = true;
@@ -263,6 +281,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(lg * 32) << 16) + buf * BN;
 #pragma unroll 1
             for (int c = 0; c < BN / 64; ++c) {        // one 32 x 64 output box per iteration
+                const int sbuf = c & (L::STAGING_BUFS - 1);   // staging boxes alternate: the store of one overlaps the next
 #pragma unroll 1
                 for (int h = 0; h < 2; ++h) {          // in two halves of 32 columns (keeps registers low)
                     const int col = c * 64 + h * 32;
@@ -299,12 +318,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                             packed[j] = pack_bf16x2(a0, a1);
                         }
                         if (h == 0) {
-                            // the previous TMA store must have finished reading the staging buffer
-                            if (lane == 0) bulk_wait_group_read<0>();
+                            // the store issued two boxes ago (same staging box) must have finished reading it
+                            if (lane == 0) bulk_wait_group_read<L::STAGING_BUFS - 1>();
                             __syncwarp();
                         }
                         // row `lane` of the 32 x 128-byte box; 16-byte chunk i lives at chunk (i ^ (row & 7))
-                        uint8_t* srow = staging_ptr + lane * 128;
+                        uint8_t* srow = staging_ptr + sbuf * L::STAGING_BOX_BYTES + lane * 128;
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
                             uint4 q = make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
@@ -316,7 +335,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     fence_proxy_async_smem();
                     __syncwarp();
                     if (lane == 0) {
-                        tma_store_2d_hint(&tm_out, staging, n0 + c * 64, m0 + lg * 32, stream_out);
+                        tma_store_2d_hint(&tm_out, staging + sbuf * L::STAGING_BOX_BYTES, n0 + c * 64, m0 + lg * 32, stream_out);
                         bulk_commit_group();
                     }
                 }
@@ -375,7 +394,7 @@ struct TcConfig {
 constexpr TcConfig kConfigs[] = {
     {"tc 128x256 per CTA, 4 stages", 1, 256, 4},
     {"tc 128x128 per CTA, 6 stages", 1, 128, 6},
-    {"tc 256x256 per CTA pair, 6 stages", 2, 256, 6},
+    {"tc 256x256 per CTA pair, 5 stages", 2, 256, 5},
     {"tc 256x128 per CTA pair, 8 stages", 2, 128, 8},
 };
 constexpr int kNumConfigs = sizeof(kConfigs) / sizeof(kConfigs[0]);
@@ -388,6 +407,14 @@ int sm_count() {
         return v > 0 ? v : 148;
     }();
     return n;
+}
+
+// Width (in tile columns) of the raster bands. W8A8_RASTER_GN overrides it for sweeps.
+int raster_band(const GemmArgs& a) {
+    static const int forced = [] { const char* e = getenv("W8A8_RASTER_GN"); return e ? atoi(e) : 0; }();
+    if (forced > 0) return forced;
+    (void)a;
+    return 1 << 20;      // along N first: measured as good as any banding, and what the from-bf16 entry needs
 }
 
 template <int CG, int BN, int STAGES, bool RAW>
@@ -433,7 +460,7 @@ int launch_cfg(const GemmArgs& a, cudaStream_t st) {
     cfg.numAttrs = na;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tm_a, tm_b, tm_out, a.s_tok, a.s_ch, a.bias,
                                        RAW ? static_cast<int32_t*>(a.out) : nullptr, a.M, a.N, a.K, a.status,
-                                       a.after_quantizer ? 1 : 0, a.flags, a.epoch, a.flags != nullptr ? 1 : 0);
+                                       a.after_quantizer ? 1 : 0, a.flags, a.epoch, raster_band(a));
     return e == cudaSuccess ? 0 : 6;
 }
 
@@ -442,7 +469,7 @@ int launch_by_id(int id, const GemmArgs& a, cudaStream_t st) {
     switch (id) {
         case 0: return launch_cfg<1, 256, 4, RAW>(a, st);
         case 1: return launch_cfg<1, 128, 6, RAW>(a, st);
-        case 2: return launch_cfg<2, 256, 6, RAW>(a, st);
+        case 2: return launch_cfg<2, 256, 5, RAW>(a, st);
         case 3: return launch_cfg<2, 128, 8, RAW>(a, st);
         default: return 1;
     }
@@ -450,10 +477,15 @@ int launch_by_id(int id, const GemmArgs& a, cudaStream_t st) {
 
 int pick_config(int M, int N, int K) {
     (void)K;
-    // small problems: more, smaller tiles fill the SMs better
-    const long tiles256 = static_cast<long>((M + BM - 1) / BM) * ((N + 255) / 256);
-    if (tiles256 < sm_count()) return 1;
-    return 0;
+    // From measurements on the five benchmark shapes: CTA pairs win once there are about two waves of
+    // 256x256 pair tiles; below that one CTA per 128x256 tile fills the SMs better; tiny problems take
+    // 128x128 tiles.
+    const long n256 = (N + 255) / 256;
+    const long pair_tiles = static_cast<long>((M + 2 * BM - 1) / (2 * BM)) * n256;
+    const long tiles256 = static_cast<long>((M + BM - 1) / BM) * n256;
+    if (pair_tiles >= 2 * (sm_count() / 2)) return 2;
+    if (tiles256 >= sm_count()) return 0;
+    return 1;
 }
 
 } // namespace
