@@ -83,8 +83,6 @@ int int8_quantize_act_per_token(const void* A_bf16, int64_t M, int64_t K, int64_
  * Bytes of caller-provided device workspace int8_linear_fused needs for this
  * problem (0 on invalid sizes). Layout, from the workspace base (which must be
  * 256-byte aligned): a 256-byte status block; then, for bf16 activations only,
- * one 64-bit progress flag per row (padded to 256 bytes; the quantizer
- * publishes finished rows there and the GEMM follows them block by block),
  * s_tok as fp32 [M] (padded to 256 bytes) and qa as int8 [M,K] dense. The
  * workspace needs no initialisation. After a bf16 call the caller may read qa
  * and s_tok back from there (int8_linear_workspace_offsets gives the offsets).
@@ -140,7 +138,7 @@ int int8_linear_fused_host(const void* A_host, void* d_A,
  * For callers that cannot provide a workspace because they cannot allocate one: a server whose own arena
  * already owns all device memory, a latency-critical loop where cudaMalloc's implicit synchronisation is
  * not acceptable, a plug-in that only ever receives its input and output buffers. The scratch that
- * int8_linear_fused takes from the caller (status word, per-row progress flags, s_tok, qa) is a fixed
+ * int8_linear_fused takes from the caller (status word, s_tok, qa) is a fixed
  * array of W8A8_STATIC_WORKSPACE_BYTES inside the library's device image; every GPU that loads the library
  * holds that much memory until the process exits. The call itself allocates nothing (no cudaMalloc,
  * cudaFree or allocating library routine).
@@ -152,14 +150,14 @@ int int8_linear_fused_host(const void* A_host, void* d_A,
  * Limits and rules:
  *   - Problems whose scratch, int8_linear_workspace_bytes(M, N, K, W8A8_ACT_BF16), exceeds
  *     W8A8_STATIC_WORKSPACE_BYTES are refused with W8A8_ERR_WORKSPACE before anything is enqueued
- *     (roughly M * (K + 12) <= 16 MiB: e.g. M = 4608 tokens at K = 3072, not at K = 12288).
+ *     (roughly M * (K + 4) <= 16 MiB: e.g. M = 4608 tokens at K = 3072, not at K = 12288).
  *   - The first call on each device looks up the array's device address (a one-time set-up step under a
  *     mutex). Make that first call outside any stream capture.
  *   - All calls on a device share the one array. Calls on the same stream run one after the other and are
  *     safe; calls that may overlap on the GPU (different streams, different host threads) race on it and
  *     must be serialized by the caller, or use int8_linear_fused with separate workspaces.
  *   - The array keeps whatever the last call left in it. Nothing needs clearing: each call resets the
- *     status word and uses a fresh progress-flag value.
+ *     status word and rewrites the scales and codes it reads.
  */
 #define W8A8_STATIC_WORKSPACE_BYTES (16u * 1024u * 1024u)
 int int8_linear_fused_static(const void* A_bf16, int64_t lda,

@@ -4,7 +4,6 @@
 #include "internal.h"
 
 #include <atomic>
-#include <random>
 #include <cstdint>
 
 namespace {
@@ -41,24 +40,10 @@ int check_dims(int64_t M, int64_t N, int64_t K) {
     return W8A8_OK;
 }
 
-// workspace for bf16 activations: [status 256 B][quantizer flags, 8 B per row][s_tok][qa]
-size_t flags_bytes(int64_t M) {
-    return round_up(static_cast<size_t>(M) * sizeof(unsigned long long), 256);
-}
+// workspace for bf16 activations: [status 256 B][s_tok, padded to 256 B][qa]
 void offsets(int64_t M, size_t* s_tok_off, size_t* qa_off) {
-    *s_tok_off = kStatusBlock + flags_bytes(M);
+    *s_tok_off = kStatusBlock;
     *qa_off = *s_tok_off + round_up(static_cast<size_t>(M) * sizeof(float), 256);
-}
-
-// A value no earlier call (and, with overwhelming probability, no uninitialised memory) has left in a
-// flag word: a random 64-bit start, incremented per call.
-unsigned long long next_epoch() {
-    static std::atomic<unsigned long long> e{[] {
-        std::random_device rd;
-        unsigned long long v = (static_cast<unsigned long long>(rd()) << 32) ^ rd();
-        return v | 1ull;
-    }()};
-    return e.fetch_add(1) + 1;
 }
 
 } // namespace
@@ -104,7 +89,7 @@ int int8_quantize_act_per_token(const void* A_bf16, int64_t M, int64_t K, int64_
     if (K % 16 != 0 || lda % 8 != 0 || !aligned16(A_bf16) || !aligned16(qa)) return W8A8_ERR_ALIGNMENT;
     if (int e = check_arch()) return e;
     cudaError_t ce = launch_quantize_bf16(A_bf16, lda, static_cast<int>(M), static_cast<int>(K), qa, s_tok, nullptr,
-                                          nullptr, 0ull, -1, static_cast<cudaStream_t>(stream));
+                                          static_cast<cudaStream_t>(stream));
     return ce == cudaSuccess ? W8A8_OK : W8A8_ERR_CUDA;
 }
 
@@ -155,18 +140,12 @@ int int8_linear_fused(const void* A, int a_dtype, int64_t lda, const float* s_to
         offsets(M, &s_off, &q_off);
         float* s_tok = reinterpret_cast<float*>(ws + s_off);
         int8_t* qa = reinterpret_cast<int8_t*>(ws + q_off);
-        const int forced_cfg = g_forced_config.load();
-        const bool skinny = (forced_cfg < 0 && M <= kSkinnyM) || forced_cfg == tc_num_configs();
-        // the tensor-core GEMM follows the quantizer row block by row block through the flags
-        unsigned long long* flags = skinny ? nullptr : reinterpret_cast<unsigned long long*>(ws + kStatusBlock);
-        const unsigned long long epoch = next_epoch();
-        const int burst_rows = skinny ? -1 : tc_first_wave_rows(g.M, g.N, g.K, forced_cfg);
-        if (launch_quantize_bf16(A, lda, g.M, g.K, qa, s_tok, status, flags, epoch, burst_rows, st) != cudaSuccess)
-            return W8A8_ERR_CUDA;
-        g.qa = qa; g.lda_q = K; g.s_tok = s_tok; g.after_quantizer = true; g.flags = flags; g.epoch = epoch;
+        // the quantizer clears the status word; the GEMM behind it (programmatic dependent launch) sets
+        // itself up while the quantizer runs and waits for it before its first read
+        if (launch_quantize_bf16(A, lda, g.M, g.K, qa, s_tok, status, st) != cudaSuccess) return W8A8_ERR_CUDA;
+        g.qa = qa; g.lda_q = K; g.s_tok = s_tok; g.after_quantizer = true;
     } else {
         g.qa = static_cast<const int8_t*>(A); g.lda_q = lda; g.s_tok = s_tok_in; g.after_quantizer = false;
-        g.epoch = next_epoch();
     }
     const int forced = g_forced_config.load();
     if ((forced < 0 && M <= kSkinnyM) || forced == tc_num_configs())
@@ -206,7 +185,7 @@ int int8_gemm_i32_debug(const int8_t* qa, const int8_t* qw, int32_t* acc,
     GemmArgs g{};
     g.qa = qa; g.lda_q = K; g.s_tok = nullptr; g.qw = qw; g.s_ch = nullptr; g.bias = nullptr;
     g.out = acc; g.ldo = N; g.M = static_cast<int>(M); g.N = static_cast<int>(N); g.K = static_cast<int>(K);
-    g.raw_i32 = true; g.status = status; g.after_quantizer = false; g.epoch = next_epoch();
+    g.raw_i32 = true; g.status = status; g.after_quantizer = false;
     const int forced = g_forced_config.load();
     if ((forced < 0 && M <= kSkinnyM) || forced == tc_num_configs())
         return launch_gemm_simt(g, st) == cudaSuccess ? W8A8_OK : W8A8_ERR_CUDA;

@@ -45,7 +45,7 @@ constexpr int NUM_THREADS = 192;
 constexpr int EPI_THREADS = 128;
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;   // 2 s
 
-enum Where { W_PRODUCER_EMPTY = 1, W_MMA_FULL = 2, W_MMA_TMEM_EMPTY = 3, W_EPI_TMEM_FULL = 4, W_DRAIN = 5, W_QUANT_FLAG = 6 };
+enum Where { W_PRODUCER_EMPTY = 1, W_MMA_FULL = 2, W_MMA_TMEM_EMPTY = 3, W_EPI_TMEM_FULL = 4, W_DRAIN = 5 };
 
 template <int CG, int BN, int STAGES>
 struct SmemLayout {
@@ -80,8 +80,7 @@ __global__ void __maxnreg__(128)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                const __grid_constant__ CUtensorMap tm_out,
                const float* __restrict__ s_tok, const float* __restrict__ s_ch, const float* __restrict__ bias,
-               int32_t* __restrict__ raw_out, int M, int N, int K, int* status, int after_quantizer,
-               const unsigned long long* __restrict__ flags, unsigned long long epoch, int raster_gn) {
+               int32_t* __restrict__ raw_out, int M, int N, int K, int* status, int after_quantizer, int raster_gn) {
     using L = SmemLayout<CG, BN, STAGES>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -144,33 +143,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         const int w = min(gn, num_n - band * gn);
         return r / w;
     };
-    // row r is quantized once flags[r] carries this call's epoch; a warp checks the BM rows of a block
-    auto rows_ready = [&](int m0, int where) {
-        bool ok = true;
-        for (int r = m0 + lane; r < min(m0 + BM, M) && ok; r += 32)
-            ok = flag_wait(flags + r, epoch, ctl, where, kStatusTimeout);
-        return __all_sync(0xffffffffu, ok) != 0;
-    };
-
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer (both CTAs of a pair)
-        if (after_quantizer && flags == nullptr && lane == 0) grid_dep_wait();   // qa comes from the kernel before this one
+        if (after_quantizer && lane == 0) grid_dep_wait();   // qa comes from the kernel before this one
         __syncwarp();
         int stage = 0;
         uint32_t phase = 0;
         int issued = 0;
         bool ok = true;
-        int ready_m0 = -1;
         for (int t = first_tile; t < num_tiles && ok; t += tile_step) {
             const int m0 = tile_m(t) * TILE_M + rank * BM;
             const int n0 = tile_n(t) * BN + rank * L::B_ROWS;
-            if (flags != nullptr && m0 != ready_m0 && m0 < M) {      // all lanes poll, one flag per row
-                if (!rows_ready(m0, W_QUANT_FLAG)) { ok = false; break; }
-                ready_m0 = m0;
-            }
             if (lane == 0) {
                 const uint64_t keep = l2_policy_evict_last();        // operands are re-read by other tiles: keep them in L2
-                if (flags != nullptr) fence_proxy_async_all();       // the TMA reads below come after the acquire
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, ctl, W_PRODUCER_EMPTY, kStatusTimeout)) { ok = false; break; }
                     const uint32_t sa = base + stage * L::STAGE_BYTES;
@@ -250,19 +235,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         uint8_t* staging_ptr = base_ptr + L::OFF_STAGING + (warp - 2) * L::STAGING_BYTES_PER_WARP;
         const bool has_bias = bias != nullptr;
         const uint64_t stream_out = l2_policy_evict_first();        // the output is written once and not read here
-        if (after_quantizer && flags == nullptr) grid_dep_wait();   // s_tok comes from the kernel before this one
+        if (after_quantizer) grid_dep_wait();          // s_tok comes from the kernel before this one
         bool ok = true;
         int it = 0;
-        int ready_m0 = -1;
         for (int t = first_tile; t < num_tiles; t += tile_step, ++it) {
             const int buf = it & 1;
             const int m0 = tile_m(t) * TILE_M + rank * BM, n0 = tile_n(t) * BN;
-            if (flags != nullptr && ok && m0 != ready_m0) {             // s_tok of this thread's row is published
-                const int r = m0 + lg * 32 + lane;
-                const bool mine = r >= M || flag_wait(flags + r, epoch, ctl, W_QUANT_FLAG, kStatusTimeout);
-                if (!__all_sync(0xffffffffu, mine)) ok = false;
-                ready_m0 = m0;
-            }
             if (!RAW_I32) {
                 asm volatile("bar.sync 1, 128;" ::: "memory");     // previous tile's readers are done
                 for (int j = ep_tid; j < BN; j += EPI_THREADS) {
@@ -344,8 +322,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         if (!RAW_I32 && lane == 0) bulk_wait_group<0>();
     }
 
-    // this grid may only count as complete once the quantizer grid before it has completed
-    if (after_quantizer && flags != nullptr && threadIdx.x == 0) grid_dep_wait();
     tc_fence_before();
     __syncthreads();
     if (CG == 2) cluster_sync_all();            // nobody leaves while the peer may still signal its barriers
@@ -460,7 +436,7 @@ int launch_cfg(const GemmArgs& a, cudaStream_t st) {
     cfg.numAttrs = na;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tm_a, tm_b, tm_out, a.s_tok, a.s_ch, a.bias,
                                        RAW ? static_cast<int32_t*>(a.out) : nullptr, a.M, a.N, a.K, a.status,
-                                       a.after_quantizer ? 1 : 0, a.flags, a.epoch, raster_band(a));
+                                       a.after_quantizer ? 1 : 0, raster_band(a));
     return e == cudaSuccess ? 0 : 6;
 }
 
@@ -492,16 +468,6 @@ int pick_config(int M, int N, int K) {
 
 int tc_num_configs() { return kNumConfigs; }
 const char* tc_config_name(int id) { return (id >= 0 && id < kNumConfigs) ? kConfigs[id].name : nullptr; }
-
-int tc_first_wave_rows(int M, int N, int K, int forced) {
-    const int id = (forced >= 0 && forced < kNumConfigs) ? forced : pick_config(M, N, K);
-    const int tile_m = BM * kConfigs[id].cg, bn = kConfigs[id].bn;
-    const int num_n = (N + bn - 1) / bn;
-    const int groups = sm_count() / kConfigs[id].cg;             // tiles in flight at once
-    const int m_blocks = (groups + num_n - 1) / num_n;          // N-fastest order: rows of that many row blocks
-    const long rows = static_cast<long>(m_blocks) * tile_m;
-    return rows < M ? static_cast<int>(rows) : M;
-}
 
 int launch_gemm_tc(const GemmArgs& a, int forced, cudaStream_t st) {
     const int id = (forced >= 0 && forced < kNumConfigs) ? forced : pick_config(a.M, a.N, a.K);

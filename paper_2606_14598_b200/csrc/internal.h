@@ -12,14 +12,9 @@ namespace w8a8 {
 constexpr int kStatusTimeout = 7;
 
 // ---- quantize.cu
-// The activation quantizer can publish one 64-bit flag per finished row (flags[row] = epoch). Rows are
-// finished in ascending order. burst_rows >= 0: after at least that many rows the kernel shrinks to one
-// CTA per SM so that a GEMM CTA fits beside it; burst_rows < 0: it keeps every SM to itself.
+// status_to_clear: workspace status word the kernel resets (or nullptr)
 cudaError_t launch_quantize_bf16(const void* A, int64_t lda, int M, int K, int8_t* qa, float* s_tok,
-                                 int* status_to_clear, unsigned long long* flags, unsigned long long epoch,
-                                 int burst_rows, cudaStream_t st);
-// rows of A the tensor-core GEMM's first wave of tiles touches (what the quantizer should produce in its burst)
-int tc_first_wave_rows(int M, int N, int K, int forced);
+                                 int* status_to_clear, cudaStream_t st);
 cudaError_t launch_quantize_f32(const float* W, int64_t ldw, int N, int K, int8_t* qw, float* s_ch, cudaStream_t st);
 
 // ---- gemm_simt.cu : CUDA-core (dp4a) path, used for skinny M and as a cross-check
@@ -36,8 +31,6 @@ struct GemmArgs {
     bool raw_i32;
     int* status;           // workspace status word
     bool after_quantizer;  // launched behind the quantizer with programmatic dependent launch
-    const unsigned long long* flags;   // per-row completion flags of the quantizer (or nullptr)
-    unsigned long long epoch;          // value a flag holds once its rows are quantized
 };
 cudaError_t launch_gemm_simt(const GemmArgs& a, cudaStream_t st);
 

@@ -69,36 +69,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const W
     return mbar_wait_slow(bar, parity, ctl, where, status_code);
 }
 
-// Bounded wait for a 64-bit flag in global memory to take the value `want` (acquire, gpu scope).
-static __device__ __noinline__ bool flag_wait_slow(const unsigned long long* flag, unsigned long long want,
-                                                   const WaitCtl& ctl, int where, int status_code) {
-    const uint64_t t0 = globaltimer_ns();
-    uint32_t spins = 0;
-    while (true) {
-        unsigned long long v;
-        asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(flag) : "memory");
-        if (v == want) return true;
-        if ((++spins & 0x3fu) == 0) {
-            if (*ctl.abort_flag) return false;
-            if (globaltimer_ns() - t0 > ctl.limit_ns) {
-                *ctl.abort_flag = 1;
-                atomicCAS(ctl.status, 0, status_code | (where << 8));
-                return false;
-            }
-        }
-        __nanosleep(64);
-    }
-}
-__device__ __forceinline__ bool flag_wait(const unsigned long long* flag, unsigned long long want,
-                                          const WaitCtl& ctl, int where, int status_code) {
-    unsigned long long v;
-    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(flag) : "memory");
-    if (v == want) return true;
-    return flag_wait_slow(flag, want, ctl, where, status_code);
-}
-// orders this thread's earlier (generic-proxy) observations before its later async-proxy (TMA) accesses
-__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
-
 // ------------------------------------------------------------------ TMA
 __device__ __forceinline__ void prefetch_tensormap(const void* tmap) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tmap)) : "memory");

@@ -1,21 +1,18 @@
 // Row-wise symmetric absmax int8 quantizer (per-token for activations,
-// per-channel for weights): HBM-bound, one pass over the row held in registers.
+// per-channel for weights): HBM-bound, every input byte is read from memory once.
 //
 //   s    = amax > 0 ? amax / 127 : 1          (IEEE division)
-//   q[k] = clamp(rne(x[k] / s), -127, 127)    (IEEE division, round half to even)
+//   q[k] = clamp(rne(x[k] / s), -127, 127)    (IEEE quotient, round half to even)
 //
-// A persistent CTA of 16 warps works on RPC = 16 / WPR rows at a time (WPR warps share one
-// row); in sweep i the CTAs of the grid together cover the consecutive rows
-// [i * grid * RPC, (i + 1) * grid * RPC), so rows finish in ascending order. A row is split into
-// 16-element chunks and every lane keeps CPL chunks in registers between the absmax pass and the
-// quantize pass, so the input is read from memory exactly once. Loads are 128-bit, the int8 codes
-// leave as one 128-bit store per chunk.
-//
-// When the caller passes a flag array, the CTA publishes, after each sweep, the call's 64-bit
-// epoch into flags[row] of the rows it finished, with release semantics. The GEMM that follows
-// (launched with programmatic dependent launch, so that it is already resident next to this
-// kernel) acquires the flags of a row block before it loads it, and so starts on the first rows
-// while later rows are still being quantized.
+// Two kernels:
+//   * quant_rows_staged_kernel (bf16 activations, the hot one): persistent CTAs stream groups of rows
+//     through a ring of shared-memory stages filled by bulk async copies (cp.async.bulk, one per row,
+//     completing on an mbarrier), several stages ahead of the warps that consume them, so that about
+//     190 KB per SM are in flight without costing registers. A row is shared by WPR warps; each warp
+//     makes two passes over its part of the row in shared memory (absmax, then quantize) with 128-bit
+//     shared-memory loads and 64-bit global stores.
+//   * quant_rows_kernel (fp32 weights, set-up; also bf16 rows too long for a stage): rows held in
+//     registers between the two passes, 128-bit global loads.
 #include "internal.h"
 #include "ptx.cuh"
 
@@ -26,69 +23,11 @@
 namespace w8a8 {
 namespace {
 
-constexpr int WARPS = 16;                 // warps per CTA
-constexpr int CPL = 3;                    // register-resident 16-element chunks per lane
-
-template <typename T> struct Chunk;       // 16 consecutive elements of a row
-
-template <> struct Chunk<__nv_bfloat16> {
-    uint4 lo, hi;                          // 8 + 8 bf16
-    __device__ __forceinline__ void load(const __nv_bfloat16* p) {
-        const uint4* q = reinterpret_cast<const uint4*>(p);
-        lo = __ldg(q);
-        hi = __ldg(q + 1);
-    }
-    __device__ __forceinline__ void zero() { lo = make_uint4(0, 0, 0, 0); hi = lo; }
-    // bf16 -> fp32 is exact: the 16 bits become the high half of the word
-    __device__ __forceinline__ void unpack(float (&f)[16]) const {
-        const uint32_t w[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            f[2 * i] = __uint_as_float(w[i] << 16);
-            f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-        }
-    }
-    __device__ __forceinline__ float absmax() const {
-        // packed bf16x2 |x| and max, then the larger half
-        const uint32_t w[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
-        __nv_bfloat162 m = __habs2(*reinterpret_cast<const __nv_bfloat162*>(&w[0]));
-#pragma unroll
-        for (int i = 1; i < 8; ++i) m = __hmax2(m, __habs2(*reinterpret_cast<const __nv_bfloat162*>(&w[i])));
-        const uint32_t mb = *reinterpret_cast<const uint32_t*>(&m);
-        return fmaxf(__uint_as_float(mb << 16), __uint_as_float(mb & 0xffff0000u));
-    }
-};
-
-template <> struct Chunk<float> {
-    float4 v[4];
-    __device__ __forceinline__ void load(const float* p) {
-        const float4* q = reinterpret_cast<const float4*>(p);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) v[i] = __ldg(q + i);
-    }
-    __device__ __forceinline__ void zero() {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-    __device__ __forceinline__ void unpack(float (&f)[16]) const {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) { f[4 * i] = v[i].x; f[4 * i + 1] = v[i].y; f[4 * i + 2] = v[i].z; f[4 * i + 3] = v[i].w; }
-    }
-    __device__ __forceinline__ float absmax() const {
-        float m = 0.f;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) m = fmaxf(fmaxf(m, fmaxf(fabsf(v[i].x), fabsf(v[i].y))), fmaxf(fabsf(v[i].z), fabsf(v[i].w)));
-        return m;
-    }
-};
+// ------------------------------------------------------------------------------------------- arithmetic
 
 // q = clamp(rne(x / s)) with the IEEE quotient, the definition.
 __device__ __forceinline__ int quant_exact(float x, float s) {
     return max(-127, min(127, __float2int_rn(__fdiv_rn(x, s))));
-}
-__device__ __forceinline__ uint32_t quant4_exact(float a, float b, float c, float d, float s) {
-    return (uint32_t(quant_exact(a, s)) & 0xffu) | ((uint32_t(quant_exact(b, s)) & 0xffu) << 8) |
-           ((uint32_t(quant_exact(c, s)) & 0xffu) << 16) | (uint32_t(quant_exact(d, s)) << 24);
 }
 
 // The IEEE quotient without a division instruction. With inv = RN(1 / s) (correctly rounded, once
@@ -127,55 +66,249 @@ __device__ __forceinline__ uint32_t quant4(float a, float b, float c, float d, c
         const uint32_t hi = __byte_perm(quant1(c, rs), quant1(d, rs), 0x0040);
         return __byte_perm(lo, hi, 0x5410);
     }
-    return quant4_exact(a, b, c, d, rs.s);
+    return (uint32_t(quant_exact(a, rs.s)) & 0xffu) | ((uint32_t(quant_exact(b, rs.s)) & 0xffu) << 8) |
+           ((uint32_t(quant_exact(c, rs.s)) & 0xffu) << 16) | (uint32_t(quant_exact(d, rs.s)) << 24);
 }
 
-template <typename T>
-__device__ __forceinline__ uint4 quant_chunk(const Chunk<T>& c, const RowScale& rs) {
-    float f[16];
-    c.unpack(f);
-    uint4 o;
-    o.x = quant4(f[0], f[1], f[2], f[3], rs);
-    o.y = quant4(f[4], f[5], f[6], f[7], rs);
-    o.z = quant4(f[8], f[9], f[10], f[11], rs);
-    o.w = quant4(f[12], f[13], f[14], f[15], rs);
-    return o;
+// |x| maximum of 8 packed bf16 values, kept packed (two running maxima)
+__device__ __forceinline__ __nv_bfloat162 absmax8(const uint4& v, __nv_bfloat162 m) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) m = __hmax2(m, __habs2(*reinterpret_cast<const __nv_bfloat162*>(&w[i])));
+    return m;
+}
+__device__ __forceinline__ float unpack_max(__nv_bfloat162 m) {
+    const uint32_t mb = *reinterpret_cast<const uint32_t*>(&m);
+    return fmaxf(__uint_as_float(mb << 16), __uint_as_float(mb & 0xffff0000u));
+}
+// Two quotients at a time with the packed fp32x2 instructions of sm_100 (each half rounds exactly like
+// the scalar instruction): same sequence as quant1 on a pair of values held in one 64-bit register.
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+struct RowScale2 {          // RowScale with its constants replicated into both halves
+    uint64_t neg_s, inv, magic;
+};
+__device__ __forceinline__ RowScale2 make_row_scale2(const RowScale& rs) {
+    return RowScale2{pack2(-rs.s, -rs.s), pack2(rs.inv, rs.inv), pack2(MAGIC, MAGIC)};
+}
+// codes of the two bf16 values of `w` in byte 0 and byte 4 of the result
+__device__ __forceinline__ uint64_t quant2(uint32_t w, const RowScale2& r2) {
+    const uint64_t x = pack2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+    const uint64_t q0 = mul2(x, r2.inv);
+    const uint64_t r0 = fma2(r2.neg_s, q0, x);
+    const uint64_t q1 = fma2(r0, r2.inv, q0);
+    const uint64_t r1 = fma2(r2.neg_s, q1, x);
+    const uint64_t q2 = fma2(r1, r2.inv, q1);
+    return add2(q2, r2.magic);
+}
+__device__ __forceinline__ uint32_t gather4(uint64_t a, uint64_t b) {   // bytes 0 and 4 of a, then of b
+    const uint32_t lo = __byte_perm(static_cast<uint32_t>(a), static_cast<uint32_t>(a >> 32), 0x0040);
+    const uint32_t hi = __byte_perm(static_cast<uint32_t>(b), static_cast<uint32_t>(b >> 32), 0x0040);
+    return __byte_perm(lo, hi, 0x5410);
+}
+// 8 packed bf16 -> 8 int8 codes (bf16 -> fp32 is exact: the 16 bits become the high half of the word)
+__device__ __forceinline__ uint2 quant8(const uint4& v, const RowScale& rs, const RowScale2& r2) {
+    if (rs.fast)
+        return make_uint2(gather4(quant2(v.x, r2), quant2(v.y, r2)), gather4(quant2(v.z, r2), quant2(v.w, r2)));
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    float f[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        f[2 * i] = __uint_as_float(w[i] << 16);
+        f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+    return make_uint2(quant4(f[0], f[1], f[2], f[3], rs), quant4(f[4], f[5], f[6], f[7], rs));
 }
 
-// WPR warps per row (a power of two <= 16). Rows with more than WPR*32*CPL chunks
-// stream the surplus twice (absmax pass, then quantize pass) from memory / L2.
-template <typename T, int WPR>
-__global__ void __launch_bounds__(WARPS * 32, sizeof(T) == 2 ? 2 : 1)   // bf16: <= 64 registers, so a GEMM CTA fits beside it
-quant_rows_kernel(const T* __restrict__ x, int64_t ld, int rows, int K,
-                  int8_t* __restrict__ q, float* __restrict__ s_out,
-                  int* status_to_clear, unsigned long long* flags, unsigned long long epoch,
-                  int burst_sweeps, int stay_ctas) {
-    // a dependent kernel (the GEMM) may become resident right away; it synchronizes through `flags`
+// ------------------------------------------------------------------------------------------- staged kernel
+
+constexpr int SG_WARPS = 16;                         // consumer warps per CTA (one more warp produces)
+constexpr int SG_THREADS = (SG_WARPS + 1) * 32;
+constexpr int SG_SMEM_BUDGET = 200 * 1024;           // ring size target
+constexpr uint64_t SG_WAIT_LIMIT_NS = 2000000000ull; // bounded waits, as everywhere
+
+__device__ __forceinline__ void bulk_load_row(uint32_t smem_dst, const void* gsrc, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_dst), "l"(reinterpret_cast<uint64_t>(gsrc)), "r"(bytes), "r"(bar) : "memory");
+}
+
+// WPR consumer warps share a row (power of two <= SG_WARPS); a stage holds RPS = SG_WARPS / WPR rows.
+template <int WPR>
+__global__ void __launch_bounds__(SG_THREADS, 1)
+quant_rows_staged_kernel(const __nv_bfloat16* __restrict__ x, int64_t ld, int rows, int K,
+                         int8_t* __restrict__ q, float* __restrict__ s_out, int* status, int num_stages) {
+    // a dependent kernel (the GEMM) may set itself up while this one runs; it waits for this grid before reading
     grid_dep_launch_dependents();
-    if (status_to_clear != nullptr && blockIdx.x == 0 && threadIdx.x == 0) *status_to_clear = 0;
+    if (status != nullptr && blockIdx.x == 0 && threadIdx.x == 0) *status = 0;
 
-    constexpr int RPC = WARPS / WPR;                 // rows a CTA works on at a time
+    constexpr int RPS = SG_WARPS / WPR;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 127u) & ~127u;
+    uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t row_bytes = static_cast<uint32_t>(K) * 2u;
+    const uint32_t stage_bytes = RPS * row_bytes;
+    // after the ring: full[num_stages], empty[num_stages], partial maxima, abort flag
+    const uint32_t bars = base + num_stages * stage_bytes;
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (num_stages + s); };
+    float* s_red = reinterpret_cast<float*>(base_ptr + num_stages * stage_bytes + 16 * num_stages);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(s_red + SG_WARPS);
+    __shared__ int dummy_status;
+    const WaitCtl ctl{abort_flag, status != nullptr ? status : &dummy_status, SG_WAIT_LIMIT_NS};
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < num_stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), SG_WARPS); }
+        *abort_flag = 0;
+        dummy_status = 0;
+        fence_mbar_init();
+    }
+    __syncthreads();
+
+    const int total_groups = (rows + RPS - 1) / RPS;          // a group = the rows of one stage
+
+    if (warp == SG_WARPS) {
+        // ---------------------------------------------------------------- producer
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            for (int g = blockIdx.x; g < total_groups; g += gridDim.x) {
+                if (!mbar_wait(empty_bar(stage), phase ^ 1u, ctl, 1, kStatusTimeout)) break;
+                const int r0 = g * RPS;
+                const int nr = min(RPS, rows - r0);
+                mbar_arrive_expect_tx(full_bar(stage), nr * row_bytes);
+                for (int r = 0; r < nr; ++r)
+                    bulk_load_row(base + stage * stage_bytes + r * row_bytes, x + static_cast<int64_t>(r0 + r) * ld,
+                                  row_bytes, full_bar(stage));
+                if (++stage == num_stages) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else {
+        // ---------------------------------------------------------------- consumers
+        const int slot = warp / WPR, part = warp % WPR;       // row of the stage, share of that row
+        const int units = K >> 3;                             // 8-element (16-byte) units per row
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        for (int g = blockIdx.x; g < total_groups; g += gridDim.x) {
+            if (ok && !mbar_wait(full_bar(stage), phase, ctl, 2, kStatusTimeout)) ok = false;
+            ok = __all_sync(0xffffffffu, ok) != 0;
+            const int row = g * RPS + slot;
+            const bool live = ok && row < rows;
+            const uint4* srow = reinterpret_cast<const uint4*>(base_ptr + stage * stage_bytes + slot * row_bytes);
+            __nv_bfloat162 m2 = __float2bfloat162_rn(0.f);
+            if (live)
+                for (int u = part * 32 + lane; u < units; u += WPR * 32) m2 = absmax8(srow[u], m2);
+            float amax = unpack_max(m2);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+            if (WPR > 1) {
+                // the WPR warps of a row exchange their partial maxima through shared memory
+                if (lane == 0) s_red[warp] = amax;
+                asm volatile("bar.sync %0, %1;" ::"r"(1 + slot), "n"(WPR * 32) : "memory");
+#pragma unroll
+                for (int w = 0; w < WPR; ++w) amax = fmaxf(amax, s_red[slot * WPR + w]);
+                asm volatile("bar.sync %0, %1;" ::"r"(1 + slot), "n"(WPR * 32) : "memory");   // s_red may be rewritten
+            }
+            if (live) {
+                const RowScale rs = make_row_scale(amax);
+                const RowScale2 r2 = make_row_scale2(rs);
+                if (part == 0 && lane == 0) s_out[row] = rs.s;
+                uint2* qrow = reinterpret_cast<uint2*>(q + static_cast<int64_t>(row) * K);
+                for (int u = part * 32 + lane; u < units; u += WPR * 32) qrow[u] = quant8(srow[u], rs, r2);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty_bar(stage));    // this warp is done with the stage
+            if (++stage == num_stages) { stage = 0; phase ^= 1u; }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------- register kernel
+
+constexpr int WARPS = 16;                 // warps per CTA
+constexpr int CPL = 3;                    // register-resident 16-element chunks per lane
+
+template <typename T> struct Chunk;       // 16 consecutive elements of a row
+
+template <> struct Chunk<__nv_bfloat16> {
+    uint4 lo, hi;                          // 8 + 8 bf16
+    __device__ __forceinline__ void load(const __nv_bfloat16* p) {
+        const uint4* q = reinterpret_cast<const uint4*>(p);
+        lo = __ldg(q);
+        hi = __ldg(q + 1);
+    }
+    __device__ __forceinline__ void zero() { lo = make_uint4(0, 0, 0, 0); hi = lo; }
+    __device__ __forceinline__ float absmax() const {
+        return unpack_max(absmax8(hi, absmax8(lo, __float2bfloat162_rn(0.f))));
+    }
+    __device__ __forceinline__ uint4 quantize(const RowScale& rs) const {
+        const RowScale2 r2 = make_row_scale2(rs);
+        const uint2 a = quant8(lo, rs, r2), b = quant8(hi, rs, r2);
+        return make_uint4(a.x, a.y, b.x, b.y);
+    }
+};
+
+template <> struct Chunk<float> {
+    float4 v[4];
+    __device__ __forceinline__ void load(const float* p) {
+        const float4* q = reinterpret_cast<const float4*>(p);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) v[i] = __ldg(q + i);
+    }
+    __device__ __forceinline__ void zero() {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    __device__ __forceinline__ float absmax() const {
+        float m = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) m = fmaxf(fmaxf(m, fmaxf(fabsf(v[i].x), fabsf(v[i].y))), fmaxf(fabsf(v[i].z), fabsf(v[i].w)));
+        return m;
+    }
+    __device__ __forceinline__ uint4 quantize(const RowScale& rs) const {
+        return make_uint4(quant4(v[0].x, v[0].y, v[0].z, v[0].w, rs), quant4(v[1].x, v[1].y, v[1].z, v[1].w, rs),
+                          quant4(v[2].x, v[2].y, v[2].z, v[2].w, rs), quant4(v[3].x, v[3].y, v[3].z, v[3].w, rs));
+    }
+};
+
+// WPR warps per row (a power of two <= 16); a CTA works on RPC = 16 / WPR rows at a time. Rows with more
+// than WPR*32*CPL chunks stream the surplus twice (absmax pass, then quantize pass) from memory / L2.
+template <typename T, int WPR>
+__global__ void __launch_bounds__(WARPS * 32, 1)
+quant_rows_kernel(const T* __restrict__ x, int64_t ld, int rows, int K,
+                  int8_t* __restrict__ q, float* __restrict__ s_out, int* status) {
+    grid_dep_launch_dependents();
+    if (status != nullptr && blockIdx.x == 0 && threadIdx.x == 0) *status = 0;
+
+    constexpr int RPC = WARPS / WPR;
     constexpr int STRIDE = WPR * 32;
     __shared__ float s_red[WARPS];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int slot = warp / WPR, w_in_row = warp % WPR;
     const int nchunks = K >> 4;
     const int c0 = w_in_row * 32 + lane;
-    // The first `burst_sweeps` sweeps are done by the whole grid; after them only the first `stay_ctas`
-    // CTAs carry on (the others leave, which makes room on their SMs for the GEMM that follows).
-    int sweep = 0;
-    int sweep_rows = gridDim.x * RPC;
-    int sweep_base = 0;
 
 #pragma unroll 1
-    for (;; ++sweep) {
-        if (sweep == burst_sweeps) {
-            if (static_cast<int>(blockIdx.x) >= stay_ctas) break;
-            sweep_rows = stay_ctas * RPC;
-        }
-        if (sweep_base >= rows) break;
-        const int base = sweep_base + blockIdx.x * RPC;
-        sweep_base += sweep_rows;
+    for (int base = blockIdx.x * RPC; base < rows; base += gridDim.x * RPC) {
         const int row = base + slot;
         const bool live = row < rows;
         const T* xr = x + static_cast<int64_t>(live ? row : 0) * ld;
@@ -210,22 +343,19 @@ quant_rows_kernel(const T* __restrict__ x, int64_t ld, int rows, int K,
 #pragma unroll
             for (int i = 0; i < CPL; ++i) {
                 const int c = c0 + i * STRIDE;
-                if (c < nchunks) *reinterpret_cast<uint4*>(qr + c * 16) = quant_chunk(reg[i], s);
+                if (c < nchunks) *reinterpret_cast<uint4*>(qr + c * 16) = reg[i].quantize(s);
             }
             for (int c = c0 + CPL * STRIDE; c < nchunks; c += STRIDE) {
                 Chunk<T> t;
                 t.load(xr + c * 16);
-                *reinterpret_cast<uint4*>(qr + c * 16) = quant_chunk(t, s);
+                *reinterpret_cast<uint4*>(qr + c * 16) = t.quantize(s);
             }
         }
-        if (flags != nullptr || WPR > 1) __syncthreads();    // stores of the sweep are done; s_red may be reused
-        if (flags != nullptr && threadIdx.x < RPC && base + threadIdx.x < rows) {
-            // every thread's stores of this sweep happen before the flags become visible
-            __threadfence();
-            asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(flags + base + threadIdx.x), "l"(epoch) : "memory");
-        }
+        if (WPR > 1) __syncthreads();    // s_red may be rewritten by the next sweep
     }
 }
+
+// ------------------------------------------------------------------------------------------- host side
 
 int sm_count() {
     static int n = [] {
@@ -238,54 +368,64 @@ int sm_count() {
 }
 
 template <typename T, int WPR>
-cudaError_t launch(const T* x, int64_t ld, int rows, int K, int8_t* q, float* s, int* status_to_clear,
-                   unsigned long long* flags, unsigned long long epoch, int burst_rows, cudaStream_t st) {
+cudaError_t launch_reg(const T* x, int64_t ld, int rows, int K, int8_t* q, float* s, int* status, cudaStream_t st) {
     constexpr int RPC = WARPS / WPR;
     const int units = (rows + RPC - 1) / RPC;
-    const int cap = sm_count() * 2;                  // two CTAs of 16 warps fill an SM's register file
+    const int cap = sm_count() * 2;
     const int grid = units < cap ? units : cap;
-    // burst_rows < 0: the whole grid does every sweep. Otherwise the full grid only produces the first
-    // burst_rows rows (at least), then one CTA per SM carries on.
-    int burst_sweeps = 1 << 30, stay = grid;
-    if (burst_rows >= 0 && grid > sm_count()) {
-        burst_sweeps = (burst_rows + grid * RPC - 1) / (grid * RPC);
-        stay = sm_count();
-    }
-    // keep the SM's L1/shared split at maximum shared memory while this kernel runs: the GEMM CTA that
-    // joins it needs almost all of it, and the split only changes on an idle SM
-    static std::once_flag once;
-    std::call_once(once, [] {
-        cudaFuncSetAttribute(quant_rows_kernel<T, WPR>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                             cudaSharedmemCarveoutMaxShared);
-    });
-    quant_rows_kernel<T, WPR><<<grid, WARPS * 32, 0, st>>>(x, ld, rows, K, q, s, status_to_clear, flags, epoch,
-                                                           burst_sweeps, stay);
+    quant_rows_kernel<T, WPR><<<grid, WARPS * 32, 0, st>>>(x, ld, rows, K, q, s, status);
     return cudaGetLastError();
 }
 
 template <typename T>
-cudaError_t dispatch(const T* x, int64_t ld, int rows, int K, int8_t* q, float* s, int* status_to_clear,
-                     unsigned long long* flags, unsigned long long epoch, int burst_rows, cudaStream_t st) {
+cudaError_t dispatch_reg(const T* x, int64_t ld, int rows, int K, int8_t* q, float* s, int* status, cudaStream_t st) {
     const int nchunks = K / 16;
     // fewest warps per row that keep the whole row in registers (<= CPL chunks per lane)
-    if (nchunks <= 32 * CPL)  return launch<T, 1>(x, ld, rows, K, q, s, status_to_clear, flags, epoch, burst_rows, st);
-    if (nchunks <= 64 * CPL)  return launch<T, 2>(x, ld, rows, K, q, s, status_to_clear, flags, epoch, burst_rows, st);
-    if (nchunks <= 128 * CPL) return launch<T, 4>(x, ld, rows, K, q, s, status_to_clear, flags, epoch, burst_rows, st);
-    if (nchunks <= 256 * CPL) return launch<T, 8>(x, ld, rows, K, q, s, status_to_clear, flags, epoch, burst_rows, st);
-    return launch<T, 16>(x, ld, rows, K, q, s, status_to_clear, flags, epoch, burst_rows, st);
+    if (nchunks <= 32 * CPL)  return launch_reg<T, 1>(x, ld, rows, K, q, s, status, st);
+    if (nchunks <= 64 * CPL)  return launch_reg<T, 2>(x, ld, rows, K, q, s, status, st);
+    if (nchunks <= 128 * CPL) return launch_reg<T, 4>(x, ld, rows, K, q, s, status, st);
+    if (nchunks <= 256 * CPL) return launch_reg<T, 8>(x, ld, rows, K, q, s, status, st);
+    return launch_reg<T, 16>(x, ld, rows, K, q, s, status, st);
+}
+
+template <int WPR>
+cudaError_t launch_staged(const __nv_bfloat16* x, int64_t ld, int rows, int K, int8_t* q, float* s, int* status,
+                          cudaStream_t st) {
+    constexpr int RPS = SG_WARPS / WPR;
+    const int stage_bytes = RPS * K * 2;
+    int num_stages = SG_SMEM_BUDGET / stage_bytes;
+    if (num_stages > 8) num_stages = 8;
+    const int groups = (rows + RPS - 1) / RPS;
+    const int smem = num_stages * stage_bytes + 16 * num_stages + SG_WARPS * 4 + 16 + 128;
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [] {
+        attr_err = cudaFuncSetAttribute(quant_rows_staged_kernel<WPR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        SG_SMEM_BUDGET + 1024);
+    });
+    if (attr_err != cudaSuccess) return attr_err;
+    const int grid = groups < sm_count() ? groups : sm_count();
+    quant_rows_staged_kernel<WPR><<<grid, SG_THREADS, smem, st>>>(x, ld, rows, K, q, s, status, num_stages);
+    return cudaGetLastError();
 }
 
 } // namespace
 
 cudaError_t launch_quantize_bf16(const void* A, int64_t lda, int M, int K, int8_t* qa, float* s_tok,
-                                 int* status_to_clear, unsigned long long* flags, unsigned long long epoch,
-                                 int burst_rows, cudaStream_t st) {
-    return dispatch<__nv_bfloat16>(static_cast<const __nv_bfloat16*>(A), lda, M, K, qa, s_tok, status_to_clear, flags,
-                                   epoch, burst_rows, st);
+                                 int* status_to_clear, cudaStream_t st) {
+    const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(A);
+    // a warp handles up to 4 KB of a row; rows of up to 64 KB (K <= 32768) go through the staged kernel
+    const int row_bytes = K * 2;
+    if (row_bytes <= 2048)  return launch_staged<1>(x, lda, M, K, qa, s_tok, status_to_clear, st);   // 16 rows per stage
+    if (row_bytes <= 8192)  return launch_staged<2>(x, lda, M, K, qa, s_tok, status_to_clear, st);   // 8 rows per stage
+    if (row_bytes <= 16384) return launch_staged<4>(x, lda, M, K, qa, s_tok, status_to_clear, st);
+    if (row_bytes <= 32768) return launch_staged<8>(x, lda, M, K, qa, s_tok, status_to_clear, st);
+    if (row_bytes <= 65536) return launch_staged<16>(x, lda, M, K, qa, s_tok, status_to_clear, st);
+    return dispatch_reg<__nv_bfloat16>(x, lda, M, K, qa, s_tok, status_to_clear, st);
 }
 
 cudaError_t launch_quantize_f32(const float* W, int64_t ldw, int N, int K, int8_t* qw, float* s_ch, cudaStream_t st) {
-    return dispatch<float>(W, ldw, N, K, qw, s_ch, nullptr, nullptr, 0ull, -1, st);
+    return dispatch_reg<float>(W, ldw, N, K, qw, s_ch, nullptr, st);
 }
 
 } // namespace w8a8

@@ -3,9 +3,8 @@
 // Some callers cannot hand this library a workspace because they cannot get one: an inference server that
 // gave all of HBM to its own arena at start-up (a later cudaMalloc fails or fragments it), a real-time loop
 // where an allocation's implicit device synchronisation is not acceptable, or a plug-in that is only ever
-// given its input and output tensors. For them the scratch the from-bf16 path needs (status word, per-row
-// progress flags, per-token scales, int8 activations) lives in a fixed array inside the library's own device
-// image. The price: every GPU that loads the library holds kStaticWorkspaceBytes until the process exits,
+// given its input and output tensors. For them the scratch the from-bf16 path needs (status word, per-token
+// scales, int8 activations) lives in a fixed array inside the library's own device image. The price: every GPU that loads the library holds kStaticWorkspaceBytes until the process exits,
 // problems whose scratch does not fit are refused, and all calls share the one array.
 #include "../../include/w8a8_linear.h"
 
@@ -54,8 +53,8 @@ extern "C" int int8_linear_fused_static(const void* A_bf16, int64_t lda,
     void* ws = nullptr;
     if (int e = static_workspace(&ws)) return e;
     // Same kernels as int8_linear_fused, with the built-in array as their scratch. Nothing in it has to be
-    // zero on entry: the call clears the status word itself and the progress flags are matched against a
-    // fresh per-call value, so whatever the previous call left behind is harmless.
+    // zero on entry: the call clears the status word itself and writes every scale and code before reading
+    // it, so whatever the previous call left behind is harmless.
     int e = int8_linear_fused(A_bf16, W8A8_ACT_BF16, lda, nullptr, qw, s_ch, bias, out_bf16, ldo, M, N, K,
                               ws, kStaticWorkspaceBytes, stream);
     if (e != W8A8_OK || !sync_and_check) return e;

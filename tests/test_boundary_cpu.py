@@ -36,12 +36,12 @@ def test_status_strings():
 
 def test_workspace_sizes():
     assert w8.int8_linear_workspace_bytes(4608, 3072, 12288, w8.ACT_INT8) == 256
-    # status block, one 8-byte flag per row (padded to 256), s_tok (padded to 256), qa
+    # status block, s_tok (padded to 256), qa
     s_off, q_off = w8.int8_linear_workspace_offsets(4608, 12288)
-    assert s_off == 256 + 4608 * 8 and q_off == s_off + 4608 * 4 and q_off % 256 == 0
+    assert s_off == 256 and q_off == s_off + 4608 * 4 and q_off % 256 == 0
     assert w8.int8_linear_workspace_bytes(4608, 3072, 12288, w8.ACT_BF16) == q_off + 4608 * 12288
     s_off, q_off = w8.int8_linear_workspace_offsets(2, 3072)
-    assert s_off == 512 and q_off == 768 and w8.int8_linear_workspace_bytes(2, 8, 3072, w8.ACT_BF16) == 768 + 6144
+    assert s_off == 256 and q_off == 512 and w8.int8_linear_workspace_bytes(2, 8, 3072, w8.ACT_BF16) == 512 + 6144
     assert w8.int8_linear_workspace_bytes(0, 8, 16) == 0
     assert w8.int8_linear_workspace_bytes(8, 8, 16, 5) == 0
 
