@@ -73,10 +73,8 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// At most 128 registers per thread: the register file then has room for a quantizer CTA (512 threads x 64
-// registers) next to this one, which is what lets the two kernels share an SM.
 template <int CG, int BN, int STAGES, bool RAW_I32>
-__global__ void __maxnreg__(128)
+__global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                const __grid_constant__ CUtensorMap tm_out,
                const float* __restrict__ s_tok, const float* __restrict__ s_ch, const float* __restrict__ bias,
@@ -257,59 +255,51 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             if (!ok) continue;                         // keep taking the named barriers, skip the work
             tc_fence_after();
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(lg * 32) << 16) + buf * BN;
-#pragma unroll 1
-            for (int c = 0; c < BN / 64; ++c) {        // one 32 x 64 output box per iteration
+            // One chunk = 32 accumulator columns of this thread's row. Two chunks make a 32 x 64 output box.
+            // The TMEM load of the next chunk is in flight while the current one is converted.
+            const uint64_t st2 = pack2(st, st);
+            auto process = [&](int cc, const uint32_t (&v)[32]) {
+                const int col = cc * 32, h = cc & 1, c = cc >> 1;
                 const int sbuf = c & (L::STAGING_BUFS - 1);   // staging boxes alternate: the store of one overlaps the next
-#pragma unroll 1
-                for (int h = 0; h < 2; ++h) {          // in two halves of 32 columns (keeps registers low)
-                    const int col = c * 64 + h * 32;
-                    uint32_t v[32];
-                    tmem_ld_32x32b_x32(t_row + col, v);
-                    tmem_wait_ld();
-                    if (c == BN / 64 - 1 && h == 1) {  // accumulator fully read: hand the buffer back
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) {
-                            if (CG == 2) mbar_arrive_cluster(mapa_shared(tempty_bar(buf), 0));
-                            else mbar_arrive(tempty_bar(buf));
-                        }
+                if (RAW_I32) {
+                    if (row < M) {
+                        int32_t* dst = raw_out + static_cast<int64_t>(row) * N + n0 + col;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (n0 + col + j < N) dst[j] = static_cast<int32_t>(v[j]);
                     }
-                    if (RAW_I32) {
-                        if (row < M) {
-                            int32_t* dst = raw_out + static_cast<int64_t>(row) * N + n0 + col;
+                } else {
+                uint32_t packed[16];
 #pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                if (n0 + col + j < N) dst[j] = static_cast<int32_t>(v[j]);
-                        }
-                    } else {
-                        uint32_t packed[16];
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const float2 sc = *reinterpret_cast<const float2*>(sm_sch + col + 2 * j);
-                            float a0 = __fmul_rn(__fmul_rn(__int2float_rn(static_cast<int>(v[2 * j])), st), sc.x);
-                            float a1 = __fmul_rn(__fmul_rn(__int2float_rn(static_cast<int>(v[2 * j + 1])), st), sc.y);
-                            if (has_bias) {
-                                const float2 bi = *reinterpret_cast<const float2*>(sm_bias + col + 2 * j);
-                                a0 = __fadd_rn(a0, bi.x);
-                                a1 = __fadd_rn(a1, bi.y);
-                            }
-                            packed[j] = pack_bf16x2(a0, a1);
-                        }
-                        if (h == 0) {
-                            // the store issued two boxes ago (same staging box) must have finished reading it
-                            if (lane == 0) bulk_wait_group_read<L::STAGING_BUFS - 1>();
-                            __syncwarp();
-                        }
-                        // row `lane` of the 32 x 128-byte box; 16-byte chunk i lives at chunk (i ^ (row & 7))
-                        uint8_t* srow = staging_ptr + sbuf * L::STAGING_BOX_BYTES + lane * 128;
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            uint4 q = make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
-                            *reinterpret_cast<uint4*>(srow + (((h * 4 + i) ^ (lane & 7)) << 4)) = q;
-                        }
+                for (int j = 0; j < 16; ++j) {
+                    // (float(acc) * s_tok) * s_ch + bias on two columns at a time; each half rounds like the scalar op
+                    uint64_t t = pack2(__int2float_rn(static_cast<int>(v[2 * j])), __int2float_rn(static_cast<int>(v[2 * j + 1])));
+                    t = mul2(t, st2);
+                    t = mul2(t, *reinterpret_cast<const uint64_t*>(sm_sch + col + 2 * j));
+                    float a0, a1;
+                    unpack2(t, a0, a1);
+                    if (has_bias) {
+                        // scalar adds: a packed add right behind the packed multiply was seen to be contracted
+                        // into a fused multiply-add by the assembler, which changes the rounding
+                        const float2 bi = *reinterpret_cast<const float2*>(sm_bias + col + 2 * j);
+                        a0 = __fadd_rn(a0, bi.x);
+                        a1 = __fadd_rn(a1, bi.y);
                     }
+                    packed[j] = pack_bf16x2(a0, a1);
                 }
-                if (!RAW_I32) {
+                if (h == 0) {
+                    // the store issued STAGING_BUFS boxes ago (same staging box) must have finished reading it
+                    if (lane == 0) bulk_wait_group_read<L::STAGING_BUFS - 1>();
+                    __syncwarp();
+                }
+                // row `lane` of the 32 x 128-byte box; 16-byte chunk i lives at chunk (i ^ (row & 7))
+                uint8_t* srow = staging_ptr + sbuf * L::STAGING_BOX_BYTES + lane * 128;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    uint4 q = make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
+                    *reinterpret_cast<uint4*>(srow + (((h * 4 + i) ^ (lane & 7)) << 4)) = q;
+                }
+                if (h == 1) {
                     fence_proxy_async_smem();
                     __syncwarp();
                     if (lane == 0) {
@@ -317,6 +307,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                         bulk_commit_group();
                     }
                 }
+                }
+            };
+            auto release_accumulator = [&]() {         // every TMEM load of this tile has completed
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    if (CG == 2) mbar_arrive_cluster(mapa_shared(tempty_bar(buf), 0));
+                    else mbar_arrive(tempty_bar(buf));
+                }
+            };
+            constexpr int CHUNKS = BN / 32;
+            uint32_t va[32], vb[32];
+            tmem_ld_32x32b_x32(t_row, va);
+#pragma unroll 1
+            for (int cc = 0; cc < CHUNKS; cc += 2) {
+                tmem_wait_ld();
+                tmem_ld_32x32b_x32(t_row + (cc + 1) * 32, vb);
+                process(cc, va);
+                tmem_wait_ld();
+                if (cc + 2 < CHUNKS) tmem_ld_32x32b_x32(t_row + (cc + 2) * 32, va);
+                else release_accumulator();
+                process(cc + 1, vb);
             }
         }
         if (!RAW_I32 && lane == 0) bulk_wait_group<0>();

@@ -81,28 +81,8 @@ __device__ __forceinline__ float unpack_max(__nv_bfloat162 m) {
     const uint32_t mb = *reinterpret_cast<const uint32_t*>(&m);
     return fmaxf(__uint_as_float(mb << 16), __uint_as_float(mb & 0xffff0000u));
 }
-// Two quotients at a time with the packed fp32x2 instructions of sm_100 (each half rounds exactly like
-// the scalar instruction): same sequence as quant1 on a pair of values held in one 64-bit register.
-__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
-    uint64_t r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
-    uint64_t r;
-    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
-__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
-    uint64_t r;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
-    return r;
-}
-__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
-    uint64_t r;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
+// Two quotients at a time with the packed fp32x2 instructions (each half rounds exactly like the scalar
+// instruction): the same sequence as quant1 on a pair of values held in one 64-bit register.
 struct RowScale2 {          // RowScale with its constants replicated into both halves
     uint64_t neg_s, inv, magic;
 };
