@@ -122,7 +122,7 @@ __device__ __forceinline__ uint2 quant8(const uint4& v, const RowScale& rs, cons
 
 constexpr int SG_WARPS = 16;                         // consumer warps per CTA (one more warp produces)
 constexpr int SG_THREADS = (SG_WARPS + 1) * 32;
-constexpr int SG_SMEM_BUDGET = 200 * 1024;           // ring size target
+constexpr int SG_SMEM_BUDGET = 200 * 1024;           // shared memory for the rings of one SM
 constexpr uint64_t SG_WAIT_LIMIT_NS = 2000000000ull; // bounded waits, as everywhere
 
 __device__ __forceinline__ void bulk_load_row(uint32_t smem_dst, const void* gsrc, uint32_t bytes, uint32_t bar) {
@@ -132,7 +132,7 @@ __device__ __forceinline__ void bulk_load_row(uint32_t smem_dst, const void* gsr
 
 // WPR consumer warps share a row (power of two <= SG_WARPS); a stage holds RPS = SG_WARPS / WPR rows.
 template <int WPR>
-__global__ void __launch_bounds__(SG_THREADS, 1)
+__global__ void __launch_bounds__(SG_THREADS, 2)
 quant_rows_staged_kernel(const __nv_bfloat16* __restrict__ x, int64_t ld, int rows, int K,
                          int8_t* __restrict__ q, float* __restrict__ s_out, int* status, int num_stages) {
     // a dependent kernel (the GEMM) may set itself up while this one runs; it waits for this grid before reading
@@ -373,9 +373,12 @@ cudaError_t launch_staged(const __nv_bfloat16* x, int64_t ld, int rows, int K, i
                           cudaStream_t st) {
     constexpr int RPS = SG_WARPS / WPR;
     const int stage_bytes = RPS * K * 2;
-    int num_stages = SG_SMEM_BUDGET / stage_bytes;
-    if (num_stages > 8) num_stages = 8;
     const int groups = (rows + RPS - 1) / RPS;
+    // With plenty of row groups two CTAs per SM (half the ring each) hide latencies better; with few, one
+    // CTA per SM with the whole ring gets more stages ahead.
+    const int ctas_per_sm = (groups >= 8 * sm_count() && SG_SMEM_BUDGET / 2 >= 2 * stage_bytes) ? 2 : 1;
+    int num_stages = SG_SMEM_BUDGET / ctas_per_sm / stage_bytes;
+    if (num_stages > 8) num_stages = 8;
     const int smem = num_stages * stage_bytes + 16 * num_stages + SG_WARPS * 4 + 16 + 128;
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
@@ -384,7 +387,8 @@ cudaError_t launch_staged(const __nv_bfloat16* x, int64_t ld, int rows, int K, i
                                         SG_SMEM_BUDGET + 1024);
     });
     if (attr_err != cudaSuccess) return attr_err;
-    const int grid = groups < sm_count() ? groups : sm_count();
+    const int cap = ctas_per_sm * sm_count();
+    const int grid = groups < cap ? groups : cap;
     quant_rows_staged_kernel<WPR><<<grid, SG_THREADS, smem, st>>>(x, ld, rows, K, q, s, status, num_stages);
     return cudaGetLastError();
 }
