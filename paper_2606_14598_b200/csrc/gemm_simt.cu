@@ -49,7 +49,8 @@ gemm_simt_kernel(const int8_t* __restrict__ qa, int64_t lda_q, const float* __re
     // weights do not depend on the quantizer: warm the first chunk before waiting for it
     if (after_quantizer) grid_dep_wait();
 
-    for (int k = lane * 16; k < K; k += 32 * 16) {
+#pragma unroll 2
+    for (int k = lane * 16; k < K; k += 32 * 16) {      // unrolled: several 512-byte slices of each weight row in flight
         uint4 w[NPW], a[MB];
 #pragma unroll
         for (int j = 0; j < NPW; ++j) w[j] = __ldg(reinterpret_cast<const uint4*>(wrow[j] + k));
@@ -110,8 +111,8 @@ cudaError_t launch(const GemmArgs& a, cudaStream_t st) {
 } // namespace
 
 cudaError_t launch_gemm_simt(const GemmArgs& a, cudaStream_t st) {
-    if (a.M <= 2) return launch<2, 4, 4>(a, st);
-    if (a.M <= 4) return launch<4, 4, 4>(a, st);
+    if (a.M <= 2) return launch<2, 8, 4>(a, st);     // 8 weight rows per warp: more bytes in flight per SM
+    if (a.M <= 4) return launch<4, 8, 4>(a, st);
     return launch<8, 4, 4>(a, st);
 }
 

@@ -47,12 +47,13 @@ constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;   // 2 s
 
 enum Where { W_PRODUCER_EMPTY = 1, W_MMA_FULL = 2, W_MMA_TMEM_EMPTY = 3, W_EPI_TMEM_FULL = 4, W_DRAIN = 5 };
 
-template <int CG, int BN, int STAGES>
+template <int CG, int BN, int STAGES, int KBS>
 struct SmemLayout {
     static constexpr int A_BYTES = BM * BK;
     static constexpr int B_ROWS = BN / CG;                          // W rows this CTA loads per tile
     static constexpr int B_BYTES = B_ROWS * BK;
-    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int KB_BYTES = A_BYTES + B_BYTES;              // one k-block: A tile + W tile of 128 bytes of K
+    static constexpr int STAGE_BYTES = KBS * KB_BYTES;              // a pipeline stage holds KBS k-blocks
     static constexpr int STAGING_BOX_BYTES = 32 * 128;             // one 32-row x 64-column bf16 box
     // two boxes alternate per epilogue warp where shared memory allows, else one
     static constexpr int STAGING_BUFS = (STAGES * STAGE_BYTES + 8 * STAGING_BOX_BYTES + 8 * BN + 1280 <= 232448) ? 2 : 1;
@@ -73,13 +74,13 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-template <int CG, int BN, int STAGES, bool RAW_I32>
+template <int CG, int BN, int STAGES, int KBS, bool RAW_I32>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                const __grid_constant__ CUtensorMap tm_out,
                const float* __restrict__ s_tok, const float* __restrict__ s_ch, const float* __restrict__ bias,
                int32_t* __restrict__ raw_out, int M, int N, int K, int* status, int after_quantizer, int raster_gn) {
-    using L = SmemLayout<CG, BN, STAGES>;
+    using L = SmemLayout<CG, BN, STAGES, KBS>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -154,19 +155,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             const int n0 = tile_n(t) * BN + rank * L::B_ROWS;
             if (lane == 0) {
                 const uint64_t keep = l2_policy_evict_last();        // operands are re-read by other tiles: keep them in L2
-                for (int kb = 0; kb < num_kb; ++kb) {
+                for (int kb = 0; kb < num_kb; kb += KBS) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, ctl, W_PRODUCER_EMPTY, kStatusTimeout)) { ok = false; break; }
-                    const uint32_t sa = base + stage * L::STAGE_BYTES;
+                    // a stage always receives all its k-blocks: those past the end of K are zero-filled by TMA
+                    // (and skipped by the MMA thread), which keeps the byte count of the barrier constant
                     if (CG == 2) {
                         // the leader's barrier counts the bytes of both CTAs
                         if (leader) mbar_arrive_expect_tx(full_bar(stage), 2 * L::STAGE_BYTES);
                         const uint32_t fb = mapa_shared(full_bar(stage), 0);
-                        tma_load_2d_pair_hint(sa, &tm_a, fb, kb * BK, m0, keep);
-                        tma_load_2d_pair_hint(sa + L::A_BYTES, &tm_b, fb, kb * BK, n0, keep);
+#pragma unroll
+                        for (int sub = 0; sub < KBS; ++sub) {
+                            const uint32_t sa = base + stage * L::STAGE_BYTES + sub * L::KB_BYTES;
+                            tma_load_2d_pair_hint(sa, &tm_a, fb, (kb + sub) * BK, m0, keep);
+                            tma_load_2d_pair_hint(sa + L::A_BYTES, &tm_b, fb, (kb + sub) * BK, n0, keep);
+                        }
                     } else {
                         mbar_arrive_expect_tx(full_bar(stage), L::STAGE_BYTES);
-                        tma_load_2d_hint(sa, &tm_a, full_bar(stage), kb * BK, m0, keep);
-                        tma_load_2d_hint(sa + L::A_BYTES, &tm_b, full_bar(stage), kb * BK, n0, keep);
+#pragma unroll
+                        for (int sub = 0; sub < KBS; ++sub) {
+                            const uint32_t sa = base + stage * L::STAGE_BYTES + sub * L::KB_BYTES;
+                            tma_load_2d_hint(sa, &tm_a, full_bar(stage), (kb + sub) * BK, m0, keep);
+                            tma_load_2d_hint(sa + L::A_BYTES, &tm_b, full_bar(stage), (kb + sub) * BK, n0, keep);
+                        }
                     }
                     ++issued;
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -198,21 +208,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 if (!mbar_wait(tempty_bar(buf), ((it >> 1) & 1) ^ 1u, ctl, W_MMA_TMEM_EMPTY, kStatusTimeout)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * BN;
-                for (int kb = 0; kb < num_kb; ++kb) {
+                for (int kb = 0; kb < num_kb; kb += KBS) {
                     if (!mbar_wait(full_bar(stage), phase, ctl, W_MMA_FULL, kStatusTimeout)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t sa = base + stage * L::STAGE_BYTES;
-                    const uint64_t da = make_kmajor_sw128_desc(sa);
-                    const uint64_t db = make_kmajor_sw128_desc(sa + L::A_BYTES);
-                    const int ksteps = min(BK, K - kb * BK + MMA_K - 1) / MMA_K;   // skip all-zero tail steps
 #pragma unroll
-                    for (int k = 0; k < BK / MMA_K; ++k) {
-                        if (k < ksteps) {   // advancing K by 32 bytes inside the swizzled row: +2 in 16-byte units
-                            if (CG == 2) mma_i8_ss_pair(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
-                            else mma_i8_ss(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                    for (int sub = 0; sub < KBS; ++sub) {
+                        const uint32_t sa = base + stage * L::STAGE_BYTES + sub * L::KB_BYTES;
+                        const uint64_t da = make_kmajor_sw128_desc(sa);
+                        const uint64_t db = make_kmajor_sw128_desc(sa + L::A_BYTES);
+                        // K steps of this k-block that hold data (0 for a k-block past the end of K)
+                        const int left = K - (kb + sub) * BK;
+                        const int ksteps = left <= 0 ? 0 : min(BK, left + MMA_K - 1) / MMA_K;
+#pragma unroll
+                        for (int k = 0; k < BK / MMA_K; ++k) {
+                            if (k < ksteps) {   // advancing K by 32 bytes inside the swizzled row: +2 in 16-byte units
+                                const uint32_t acc = (kb | sub | k) != 0 ? 1u : 0u;
+                                if (CG == 2) mma_i8_ss_pair(d_tmem, da + 2 * k, db + 2 * k, idesc, acc);
+                                else mma_i8_ss(d_tmem, da + 2 * k, db + 2 * k, idesc, acc);
+                            }
                         }
                     }
-                    // the stage is free (in both CTAs) once these MMAs have read it
+                    // the stage is free (in both CTAs) once these MMAs have read it. One commit per stage, not per
+                    // k-block: with 128-byte stages the commits and barrier round trips cost ~8% of the run time
                     if (CG == 2) { tc_commit_pair(empty_bar(stage)); tc_commit_pair(mapa_shared(empty_bar(stage), 1)); }
                     else tc_commit(empty_bar(stage));
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -377,13 +394,15 @@ bool encode_2d(CUtensorMap* tm, CUtensorMapDataType dt, const void* ptr, uint64_
 
 struct TcConfig {
     const char* name;
-    int cg, bn, stages;
+    int cg, bn, stages, kbs;
 };
 constexpr TcConfig kConfigs[] = {
-    {"tc 128x256 per CTA, 4 stages", 1, 256, 4},
-    {"tc 128x128 per CTA, 6 stages", 1, 128, 6},
-    {"tc 256x256 per CTA pair, 5 stages", 2, 256, 5},
-    {"tc 256x128 per CTA pair, 8 stages", 2, 128, 8},
+    // measured on the c4 shapes (hot L2): pair 3 x 256 B: 117 / 111 us; pair 5 x 128 B: 125 / 120 us;
+    // pair 2 x 384 B: 127 / 131 us; one CTA 4 x 128 B: 131 / 124 us; one CTA 2 x 256 B: 144 / 136 us
+    {"tc 128x256 per CTA, 4 stages x 128 B of K", 1, 256, 4, 1},
+    {"tc 128x128 per CTA, 3 stages x 256 B of K", 1, 128, 3, 2},
+    {"tc 256x256 per CTA pair, 3 stages x 256 B of K", 2, 256, 3, 2},
+    {"tc 256x128 per CTA pair, 4 stages x 256 B of K", 2, 128, 4, 2},
 };
 constexpr int kNumConfigs = sizeof(kConfigs) / sizeof(kConfigs[0]);
 
@@ -405,11 +424,11 @@ int raster_band(const GemmArgs& a) {
     return 1 << 20;      // along N first: measured as good as any banding, and what the from-bf16 entry needs
 }
 
-template <int CG, int BN, int STAGES, bool RAW>
+template <int CG, int BN, int STAGES, int KBS, bool RAW>
 int launch_cfg(const GemmArgs& a, cudaStream_t st) {
-    using L = SmemLayout<CG, BN, STAGES>;
+    using L = SmemLayout<CG, BN, STAGES, KBS>;
     static_assert(L::DYN_BYTES <= 232448, "shared memory budget");
-    auto kern = gemm_tc_kernel<CG, BN, STAGES, RAW>;
+    auto kern = gemm_tc_kernel<CG, BN, STAGES, KBS, RAW>;
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [&] { attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES); });
@@ -455,10 +474,10 @@ int launch_cfg(const GemmArgs& a, cudaStream_t st) {
 template <bool RAW>
 int launch_by_id(int id, const GemmArgs& a, cudaStream_t st) {
     switch (id) {
-        case 0: return launch_cfg<1, 256, 4, RAW>(a, st);
-        case 1: return launch_cfg<1, 128, 6, RAW>(a, st);
-        case 2: return launch_cfg<2, 256, 5, RAW>(a, st);
-        case 3: return launch_cfg<2, 128, 8, RAW>(a, st);
+        case 0: return launch_cfg<1, 256, 4, 1, RAW>(a, st);
+        case 1: return launch_cfg<1, 128, 3, 2, RAW>(a, st);
+        case 2: return launch_cfg<2, 256, 3, 2, RAW>(a, st);
+        case 3: return launch_cfg<2, 128, 4, 2, RAW>(a, st);
         default: return 1;
     }
 }
