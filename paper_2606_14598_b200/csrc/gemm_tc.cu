@@ -61,8 +61,10 @@ struct SmemLayout {
     static constexpr int OFF_STAGING = STAGES * STAGE_BYTES;
     static constexpr int OFF_SCH = OFF_STAGING + 4 * STAGING_BYTES_PER_WARP;
     static constexpr int OFF_BIAS = OFF_SCH + BN * 4;
-    static constexpr int OFF_BARS = OFF_BIAS + BN * 4;             // full[STAGES], empty[STAGES], tfull[2], tempty[2]
-    static constexpr int NUM_BARS = 2 * STAGES + 4;
+    // full[STAGES * KBS] (one per k-block), empty[STAGES] (one per stage), tfull[2], tempty[2]
+    static constexpr int OFF_BARS = OFF_BIAS + BN * 4;
+    static constexpr int NUM_FULL = STAGES * KBS;
+    static constexpr int NUM_BARS = NUM_FULL + STAGES + 4;
     static constexpr int OFF_TMEM = OFF_BARS + NUM_BARS * 8;
     static constexpr int OFF_ABORT = OFF_TMEM + 4;
     static constexpr int TOTAL = OFF_ABORT + 4;
@@ -89,10 +91,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     const uint32_t rank = CG == 2 ? cluster_ctarank() : 0u;     // position in the CTA pair; 0 leads
     const bool leader = rank == 0;
     const uint32_t bars = base + L::OFF_BARS;
-    auto full_bar = [&](int s) { return bars + 8u * s; };                      // used in the leader
-    auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };          // one per CTA
-    auto tfull_bar = [&](int b) { return bars + 8u * (2 * STAGES + b); };      // one per CTA
-    auto tempty_bar = [&](int b) { return bars + 8u * (2 * STAGES + 2 + b); }; // used in the leader
+    // Operands arrive per k-block (the MMAs of a k-block start as soon as its 128 bytes of K have landed);
+    // shared memory is handed back per stage of KBS k-blocks (one tcgen05.commit per stage).
+    auto full_bar = [&](int s, int sub) { return bars + 8u * (s * KBS + sub); };          // used in the leader
+    auto empty_bar = [&](int s) { return bars + 8u * (L::NUM_FULL + s); };                // one per CTA
+    auto tfull_bar = [&](int b) { return bars + 8u * (L::NUM_FULL + STAGES + b); };       // one per CTA
+    auto tempty_bar = [&](int b) { return bars + 8u * (L::NUM_FULL + STAGES + 2 + b); };  // used in the leader
     volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(base_ptr + L::OFF_TMEM);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::OFF_ABORT);
     const WaitCtl ctl{abort_flag, status, WAIT_LIMIT_NS};
@@ -103,7 +107,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     // can only be recorded seconds later
     if (!after_quantizer && blockIdx.x == 0 && threadIdx.x == 0) *status = 0;
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int s = 0; s < STAGES; ++s) {
+            for (int sub = 0; sub < KBS; ++sub) mbar_init(full_bar(s, sub), 1);
+            mbar_init(empty_bar(s), 1);
+        }
         for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4 * CG); }
         *abort_flag = 0;
         fence_mbar_init();
@@ -159,23 +166,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, ctl, W_PRODUCER_EMPTY, kStatusTimeout)) { ok = false; break; }
                     // a stage always receives all its k-blocks: those past the end of K are zero-filled by TMA
                     // (and skipped by the MMA thread), which keeps the byte count of the barrier constant
-                    if (CG == 2) {
-                        // the leader's barrier counts the bytes of both CTAs
-                        if (leader) mbar_arrive_expect_tx(full_bar(stage), 2 * L::STAGE_BYTES);
-                        const uint32_t fb = mapa_shared(full_bar(stage), 0);
 #pragma unroll
-                        for (int sub = 0; sub < KBS; ++sub) {
-                            const uint32_t sa = base + stage * L::STAGE_BYTES + sub * L::KB_BYTES;
+                    for (int sub = 0; sub < KBS; ++sub) {
+                        const uint32_t sa = base + stage * L::STAGE_BYTES + sub * L::KB_BYTES;
+                        if (CG == 2) {
+                            // the leader's barrier counts the bytes of both CTAs
+                            if (leader) mbar_arrive_expect_tx(full_bar(stage, sub), 2 * L::KB_BYTES);
+                            const uint32_t fb = mapa_shared(full_bar(stage, sub), 0);
                             tma_load_2d_pair_hint(sa, &tm_a, fb, (kb + sub) * BK, m0, keep);
                             tma_load_2d_pair_hint(sa + L::A_BYTES, &tm_b, fb, (kb + sub) * BK, n0, keep);
-                        }
-                    } else {
-                        mbar_arrive_expect_tx(full_bar(stage), L::STAGE_BYTES);
-#pragma unroll
-                        for (int sub = 0; sub < KBS; ++sub) {
-                            const uint32_t sa = base + stage * L::STAGE_BYTES + sub * L::KB_BYTES;
-                            tma_load_2d_hint(sa, &tm_a, full_bar(stage), (kb + sub) * BK, m0, keep);
-                            tma_load_2d_hint(sa + L::A_BYTES, &tm_b, full_bar(stage), (kb + sub) * BK, n0, keep);
+                        } else {
+                            mbar_arrive_expect_tx(full_bar(stage, sub), L::KB_BYTES);
+                            tma_load_2d_hint(sa, &tm_a, full_bar(stage, sub), (kb + sub) * BK, m0, keep);
+                            tma_load_2d_hint(sa + L::A_BYTES, &tm_b, full_bar(stage, sub), (kb + sub) * BK, n0, keep);
                         }
                     }
                     ++issued;
@@ -192,7 +195,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 if (s == 0) { s = STAGES; ph ^= 1u; }
                 --s;
                 const uint64_t t0 = globaltimer_ns();
-                while (!mbar_try_wait(full_bar(s), ph) && globaltimer_ns() - t0 < 10000000ull) {}
+                while (!mbar_try_wait(full_bar(s, KBS - 1), ph) && globaltimer_ns() - t0 < 10000000ull) {}
             }
         }
     } else if (warp == 1) {
@@ -209,10 +212,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * BN;
                 for (int kb = 0; kb < num_kb; kb += KBS) {
-                    if (!mbar_wait(full_bar(stage), phase, ctl, W_MMA_FULL, kStatusTimeout)) { ok = false; break; }
-                    tc_fence_after();
 #pragma unroll
                     for (int sub = 0; sub < KBS; ++sub) {
+                        if (!mbar_wait(full_bar(stage, sub), phase, ctl, W_MMA_FULL, kStatusTimeout)) { ok = false; break; }
+                        tc_fence_after();
                         const uint32_t sa = base + stage * L::STAGE_BYTES + sub * L::KB_BYTES;
                         const uint64_t da = make_kmajor_sw128_desc(sa);
                         const uint64_t db = make_kmajor_sw128_desc(sa + L::A_BYTES);
@@ -228,6 +231,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                             }
                         }
                     }
+                    if (!ok) break;
                     // the stage is free (in both CTAs) once these MMAs have read it. One commit per stage, not per
                     // k-block: with 128-byte stages the commits and barrier round trips cost ~8% of the run time
                     if (CG == 2) { tc_commit_pair(empty_bar(stage)); tc_commit_pair(mapa_shared(empty_bar(stage), 1)); }
