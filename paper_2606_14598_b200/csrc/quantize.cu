@@ -195,8 +195,10 @@ quant_rows_staged_kernel(const __nv_bfloat16* __restrict__ x, int64_t ld, int ro
             const bool live = ok && row < rows;
             const uint4* srow = reinterpret_cast<const uint4*>(base_ptr + stage * stage_bytes + slot * row_bytes);
             __nv_bfloat162 m2 = __float2bfloat162_rn(0.f);
-            if (live)
+            if (live) {
+#pragma unroll 3
                 for (int u = part * 32 + lane; u < units; u += WPR * 32) m2 = absmax8(srow[u], m2);
+            }
             float amax = unpack_max(m2);
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
@@ -213,6 +215,7 @@ quant_rows_staged_kernel(const __nv_bfloat16* __restrict__ x, int64_t ld, int ro
                 const RowScale2 r2 = make_row_scale2(rs);
                 if (part == 0 && lane == 0) s_out[row] = rs.s;
                 uint2* qrow = reinterpret_cast<uint2*>(q + static_cast<int64_t>(row) * K);
+#pragma unroll 3
                 for (int u = part * 32 + lane; u < units; u += WPR * 32) qrow[u] = quant8(srow[u], rs, r2);
             }
             __syncwarp();
