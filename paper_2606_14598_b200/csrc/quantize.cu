@@ -382,6 +382,8 @@ cudaError_t launch_staged(const __nv_bfloat16* x, int64_t ld, int rows, int K, i
     const int ctas_per_sm = (groups >= 8 * sm_count() && SG_SMEM_BUDGET / 2 >= 2 * stage_bytes) ? 2 : 1;
     int num_stages = SG_SMEM_BUDGET / ctas_per_sm / stage_bytes;
     if (num_stages > 8) num_stages = 8;
+    // the ring indices of the kernel wrap at num_stages: a ring of fewer than two stages must never be launched
+    if (num_stages < 2) return cudaErrorInvalidConfiguration;
     const int smem = num_stages * stage_bytes + 16 * num_stages + SG_WARPS * 4 + 16 + 128;
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
@@ -401,7 +403,8 @@ cudaError_t launch_staged(const __nv_bfloat16* x, int64_t ld, int rows, int K, i
 cudaError_t launch_quantize_bf16(const void* A, int64_t lda, int M, int K, int8_t* qa, float* s_tok,
                                  int* status_to_clear, cudaStream_t st) {
     const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(A);
-    // a warp handles up to 4 KB of a row; rows of up to 64 KB (K <= 32768) go through the staged kernel
+    // a warp handles up to 4 KB of a row (measured best among 1-16 KB); rows of up to 64 KB (K <= 32768) go
+    // through the staged kernel, longer ones through the register kernel
     const int row_bytes = K * 2;
     if (row_bytes <= 2048)  return launch_staged<1>(x, lda, M, K, qa, s_tok, status_to_clear, st);   // 16 rows per stage
     if (row_bytes <= 8192)  return launch_staged<2>(x, lda, M, K, qa, s_tok, status_to_clear, st);   // 8 rows per stage
