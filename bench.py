@@ -27,8 +27,8 @@ if ROOT not in sys.path:
 
 METRIC = "fused W8A8 linear TOPS (% of B200 dense INT8 peak) per DiT GEMM shape"
 INT8_PEAK_TOPS = 4500.0            # B200 datasheet, dense INT8
-# measured DRAM traffic of one gemm_tc_kernel launch (ncu, see profiles/): c4 = mean of up (138.2 MB) and down (137.0 MB)
-NCU_GEMM_DRAM_BYTES_PER_LAUNCH = {"c4": 137.6e6}
+# measured DRAM traffic of one gemm_tc_kernel launch (ncu, see profiles/): c4 = mean of up (137.8 MB) and down (138.3 MB)
+NCU_GEMM_DRAM_BYTES_PER_LAUNCH = {"c4": 138.05e6}
 L2_BYTES = 126 * 1024 * 1024
 
 
@@ -193,7 +193,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--workload", default="c4", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--workload", default="c4", choices=["c1", "c2", "c3", "c4", "c5", "paper"])
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--sets", type=int, default=3, help="rotating input/weight sets (keeps steps out of L2)")
     ap.add_argument("--no-extras", action="store_true", help="skip e2e, context and CPU-baseline legs")
@@ -415,8 +415,12 @@ def main():
                 s_off, q_off = w8.int8_linear_workspace_offsets(spec.M, spec.K)
                 qa = L["ws"][q_off:q_off + spec.M * spec.K].view(torch.int8).view(spec.M, spec.K)
                 ti = statistics.mean(cuda_timer(torch, lambda: torch._int_mm(qa, L["qw"].t()), 10, 3))
+                mine = next(p for p in per_shape if p["name"] == spec.name)
                 ctx.append({"name": spec.name, "torch_bf16_matmul_tflops": spec.ops / tb / 1e12,
-                            "torch_int_mm_tops_no_dequant": spec.ops / ti / 1e12})
+                            "torch_int_mm_tops_no_dequant": spec.ops / ti / 1e12,
+                            # the paper's Table 1 quantity on this machine: fused int8 linear over library bf16 matmul
+                            "fused_from_bf16_speedup_over_bf16_matmul": tb / (mine["fused_from_bf16_us"] * 1e-6),
+                            "gemm_epilogue_speedup_over_bf16_matmul": tb / (mine["gemm_epilogue_us"] * 1e-6)})
                 del Wb
             line["context"] = ctx
 

@@ -56,6 +56,13 @@ CONFIGS: dict[str, list[LinearSpec]] = {
            LinearSpec("c5_mlp_up", 9216, 3072, 12288),
            LinearSpec("c5_mlp_down", 9216, 12288, 3072, act="gelu", outlier_frac=0.0),
            LinearSpec("c5_adaln", 2, 3072, 18432, outlier_frac=0.0)],
+    # The paper's own model (Method, "Target architecture": hidden 4608, MLP 12288, five distinct GEMM shapes
+    # (N, K)) at the in-model token count of 1024px (Results: M ~ 4110), rounded up to a multiple of 2.
+    "paper": [LinearSpec("paper_qkv", 4110, 4608, 13824),
+              LinearSpec("paper_attn_out", 4110, 4608, 4608),
+              LinearSpec("paper_ffn_up", 4110, 4608, 12288),
+              LinearSpec("paper_ffn_down", 4110, 12288, 4608, act="gelu", outlier_frac=0.0),
+              LinearSpec("paper_llm_proj", 4110, 53248, 4608)],
 }
 
 

@@ -305,7 +305,7 @@ def sample_rows(M, n=48):
     return np.array(sorted({r for r in fixed + extra if 0 <= r < M}), dtype=np.int64)
 
 
-ALL_SPECS = [s for name in ("c1", "c2", "c3", "c4", "c5") for s in synth.CONFIGS[name]]
+ALL_SPECS = [s for name in ("c1", "c2", "c3", "c4", "c5", "paper") for s in synth.CONFIGS[name]]
 
 
 @pytest.mark.parametrize("spec", ALL_SPECS, ids=[s.name for s in ALL_SPECS])
