@@ -51,6 +51,10 @@ def _load():
         lib.oracle_quantize_weight_per_channel.restype = None
         lib.oracle_quantize_act_per_token.argtypes = [vp, i64, i64, i64, vp, vp]
         lib.oracle_quantize_act_per_token.restype = None
+        lib.oracle_quantize_weight_per_channel_smooth.argtypes = [vp, i64, i64, i64, vp, vp, vp]
+        lib.oracle_quantize_weight_per_channel_smooth.restype = None
+        lib.oracle_quantize_act_per_token_smooth.argtypes = [vp, i64, i64, i64, vp, vp, vp]
+        lib.oracle_quantize_act_per_token_smooth.restype = None
         lib.oracle_gemm_i32.argtypes = [vp, vp, vp, i64, i64, i64]
         lib.oracle_gemm_i32.restype = i64
         lib.oracle_epilogue.argtypes = [vp, vp, vp, vp, vp, i64, i64]
@@ -96,6 +100,38 @@ def quantize_act_per_token(A_bits: np.ndarray):
     s_tok = np.empty((M,), np.float32)
     _load().oracle_quantize_act_per_token(_p(A_bits), M, K, K, _p(qa), _p(s_tok))
     return qa, s_tok
+
+
+def quantize_weight_per_channel_smooth(W: np.ndarray, mult: np.ndarray):
+    """fp32 [N,K] times a per-input-channel factor fp32 [K], then quantized per channel."""
+    W = _chk(W, np.float32, 2)
+    mult = _chk(mult, np.float32, 1)
+    N, K = W.shape
+    assert mult.shape == (K,)
+    qw = np.empty((N, K), np.int8)
+    s_ch = np.empty((N,), np.float32)
+    _load().oracle_quantize_weight_per_channel_smooth(_p(W), N, K, K, _p(mult), _p(qw), _p(s_ch))
+    return qw, s_ch
+
+
+def quantize_act_per_token_smooth(A_bits: np.ndarray, mult: np.ndarray):
+    """bf16 bit patterns [M,K] times a per-input-channel factor fp32 [K], then quantized per token."""
+    A_bits = _chk(A_bits, np.uint16, 2)
+    mult = _chk(mult, np.float32, 1)
+    M, K = A_bits.shape
+    assert mult.shape == (K,)
+    qa = np.empty((M, K), np.int8)
+    s_tok = np.empty((M,), np.float32)
+    _load().oracle_quantize_act_per_token_smooth(_p(A_bits), M, K, K, _p(mult), _p(qa), _p(s_tok))
+    return qa, s_tok
+
+
+def linear_fused_bf16_smooth(A_bits, a_mult, qw, s_ch, bias):
+    """Whole path from bf16 activations smoothed by a_mult. Returns dict(out, qa, s_tok, acc)."""
+    qa, s_tok = quantize_act_per_token_smooth(A_bits, a_mult)
+    r = linear_fused_int8(qa, s_tok, qw, s_ch, bias)
+    r.update(qa=qa, s_tok=s_tok)
+    return r
 
 
 def gemm_i32(qa: np.ndarray, qw: np.ndarray) -> np.ndarray:

@@ -95,6 +95,35 @@ void oracle_quantize_weight_per_channel(const float* W, int64_t N, int64_t K, in
         quant_row(W + n * ldw, K, qw + n * K, s_ch + n);
 }
 
+// SmoothQuant hook (the paper's recipe names SmoothQuant, alpha = 0.5; Method, "The quantization recipe"):
+// a per-input-channel factor is multiplied into the operand before quantization, x'[k] = x[k] * mult[k]
+// (one fp32 multiply, rounded), activations by 1/s_k and weights by s_k, so that the product is unchanged.
+// How s is calibrated is outside this path; the factors are inputs. mult == NULL means no smoothing.
+void oracle_quantize_weight_per_channel_smooth(const float* W, int64_t N, int64_t K, int64_t ldw, const float* mult,
+                                               int8_t* qw, float* s_ch) {
+    #pragma omp parallel for schedule(static)
+    for (int64_t n = 0; n < N; ++n) {
+        float* row = new float[K > 0 ? K : 1];
+        for (int64_t k = 0; k < K; ++k) row[k] = mult ? W[n * ldw + k] * mult[k] : W[n * ldw + k];
+        quant_row(row, K, qw + n * K, s_ch + n);
+        delete[] row;
+    }
+}
+
+void oracle_quantize_act_per_token_smooth(const uint16_t* A, int64_t M, int64_t K, int64_t lda, const float* mult,
+                                          int8_t* qa, float* s_tok) {
+    #pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m) {
+        float* row = new float[K > 0 ? K : 1];
+        for (int64_t k = 0; k < K; ++k) {
+            const float x = bf16_to_f32(A[m * lda + k]);
+            row[k] = mult ? x * mult[k] : x;
+        }
+        quant_row(row, K, qa + m * K, s_tok + m);
+        delete[] row;
+    }
+}
+
 // Per-token activation quantization. A is bf16 (raw 16-bit patterns) [M, K]
 // with row stride lda (elements); qa is int8 [M, K] dense; s_tok is fp32 [M].
 void oracle_quantize_act_per_token(const uint16_t* A, int64_t M, int64_t K, int64_t lda,

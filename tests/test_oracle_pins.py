@@ -359,3 +359,58 @@ def test_generator_is_seeded_and_shaped():
     assert std[torch.from_numpy(mask)].mean() > 15 and std[torch.from_numpy(~mask)].mean() < 1.3
     g = synth.make_activations(synth.LinearSpec("g", 64, 1024, 8, act="gelu", outlier_frac=0.0))
     assert g.float().min() > -0.18 and g.float().max() > 2.0
+
+
+# --------------------------------------------------------------------------- SmoothQuant hook
+
+def test_smooth_ones_is_plain_and_powers_of_two_are_exact():
+    rng = np.random.default_rng(12)
+    a = rng.standard_normal((24, 160)).astype(np.float32)
+    a[:, 5] *= 20
+    bits = bf16_bits_of(a)
+    ones = np.ones(160, np.float32)
+    q0, s0 = oracle.quantize_act_per_token(bits)
+    q1, s1 = oracle.quantize_act_per_token_smooth(bits, ones)
+    assert (q0 == q1).all() and (s0 == s1).all()
+    # a power-of-two factor per input channel multiplies exactly: the result must equal quantizing the
+    # exactly scaled matrix (built here in float64). This pins that the factor is indexed by k (not by row)
+    # and applied before the absmax.
+    e = rng.integers(-3, 4, 160)
+    mult = np.ldexp(np.ones(160), e).astype(np.float32)
+    scaled = (bits_to_f64(bits) * np.ldexp(1.0, e)[None, :]).astype(np.float32)
+    q2, s2 = oracle.quantize_act_per_token_smooth(bits, mult)
+    q3, s3 = oracle.quantize_weight_per_channel(scaled)
+    assert (q2 == q3).all() and (s2 == s3).all()
+    assert (q2 != q0).any()
+    W = (rng.standard_normal((16, 160)) * 0.02).astype(np.float32)
+    qw2, sw2 = oracle.quantize_weight_per_channel_smooth(W, mult)
+    qw3, sw3 = oracle.quantize_weight_per_channel((W.astype(np.float64) * np.ldexp(1.0, e)[None, :]).astype(np.float32))
+    assert (qw2 == qw3).all() and (sw2 == sw3).all()
+    # general factors: one rounded fp32 multiply per element (float64 product of two float32 values is exact)
+    m = (rng.random(160) * 3 + 0.1).astype(np.float32)
+    xs = (bits_to_f64(bits) * m.astype(np.float64)[None, :]).astype(np.float32)
+    q4, s4 = oracle.quantize_act_per_token_smooth(bits, m)
+    q5, s5 = oracle.quantize_weight_per_channel(xs)
+    assert (q4 == q5).all() and (s4 == s5).all()
+
+
+def test_smoothing_keeps_the_product_and_tames_outlier_channels():
+    """X diag(1/s) (diag(s) W)^T = X W^T, so the smoothed path approximates the same float matmul; with
+    s_k = sqrt(max|X_k| / max|W_k|) (alpha = 0.5) the outlier channels stop dominating the per-token scales
+    and the error drops."""
+    spec = synth.LinearSpec("smooth", 96, 1024, 128, outlier_frac=0.02, outlier_mult=20.0)
+    t = synth.make_linear(spec)
+    A_bits = synth.bf16_bits(t["A"])
+    W, b = t["W"].numpy(), t["bias"].numpy()
+    ref = float_linear(A_bits, W, b)
+    qw, s_ch = oracle.quantize_weight_per_channel(W)
+    plain = bits_to_f64(oracle.linear_fused_bf16(A_bits, qw, s_ch, b)["out"])
+    ax = np.abs(bits_to_f64(A_bits)).max(axis=0)
+    aw = np.abs(W.astype(np.float64)).max(axis=0)
+    s = np.sqrt(ax / aw)
+    a_mult, w_mult = (1.0 / s).astype(np.float32), s.astype(np.float32)
+    qw_s, s_ch_s = oracle.quantize_weight_per_channel_smooth(W, w_mult)
+    smooth = bits_to_f64(oracle.linear_fused_bf16_smooth(A_bits, a_mult, qw_s, s_ch_s, b)["out"])
+    err_plain = np.linalg.norm(plain - ref) / np.linalg.norm(ref)
+    err_smooth = np.linalg.norm(smooth - ref) / np.linalg.norm(ref)
+    assert err_smooth < 0.6 * err_plain and err_smooth < 0.03, (err_plain, err_smooth)
