@@ -118,6 +118,25 @@ int int8_linear_fused(const void* A, int a_dtype, int64_t lda, const float* s_to
                       void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * SmoothQuant hook (Method, "The quantization recipe (reused)": the recipe is W8A8 with SmoothQuant,
+ * alpha = 0.5). A per-input-channel factor is multiplied into the operand before it is quantized:
+ *     x'[m,k] = float(A[m,k]) * a_mult[k]      W'[n,k] = W[n,k] * w_mult[k]      (one rounded fp32 multiply)
+ * and everything else is as in the plain entry points applied to x' / W'. With a_mult = 1/s and w_mult = s the
+ * product is unchanged and outlier channels of the activations are tamed; how s is calibrated (the paper uses
+ * s_k = max|X_k|^0.5 / max|W_k|^0.5 over a calibration set) is the caller's business: the factors are inputs.
+ *   a_mult / w_mult  in  fp32 [K], device, 16-byte aligned, required (use the plain entry points for none)
+ * All other arguments, requirements and errors as for the entry point without the suffix.
+ */
+int int8_quantize_weight_per_channel_smooth(const float* W, int64_t N, int64_t K, int64_t ldw, const float* w_mult,
+                                            int8_t* qw, float* s_ch, void* stream);
+int int8_quantize_act_per_token_smooth(const void* A_bf16, int64_t M, int64_t K, int64_t lda, const float* a_mult,
+                                       int8_t* qa, float* s_tok, void* stream);
+int int8_linear_fused_smooth(const void* A_bf16, int64_t lda, const float* a_mult,
+                             const int8_t* qw, const float* s_ch, const float* bias,
+                             void* out_bf16, int64_t ldo, int64_t M, int64_t N, int64_t K,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Same computation with the activations and the result in HOST memory
  * (pinned memory makes the copies asynchronous): copies A to d_A, runs
  * int8_linear_fused on bf16 activations, copies the result to out_host, all on

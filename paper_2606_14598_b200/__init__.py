@@ -8,5 +8,6 @@ from .binding import (  # noqa: F401
     ACT_BF16, ACT_INT8, K_MAX, W8A8Error, alloc_workspace, config_name, force_config, int8_check_status,
     int8_gemm_i32_debug, int8_linear_fused, int8_linear_fused_host, int8_linear_fused_static, int8_linear_workspace_bytes,
     int8_linear_workspace_offsets, int8_quantize_act_per_token, int8_quantize_weight_per_channel, num_configs,
+    int8_quantize_act_per_token_smooth, int8_quantize_weight_per_channel_smooth, int8_linear_fused_smooth,
     status_string,
 )

@@ -25,7 +25,8 @@ EXPORTS = (
     "int8_quantize_weight_per_channel", "int8_quantize_act_per_token", "int8_linear_workspace_bytes",
     "int8_linear_workspace_offsets", "int8_linear_fused", "int8_linear_fused_host", "int8_gemm_i32_debug",
     "int8_check_status", "int8_linear_force_config", "int8_linear_num_configs", "int8_linear_config_name",
-    "int8_status_string", "int8_linear_fused_static",
+    "int8_status_string", "int8_linear_fused_static", "int8_quantize_weight_per_channel_smooth",
+    "int8_quantize_act_per_token_smooth", "int8_linear_fused_smooth",
 )
 
 if not os.path.exists(LIB_PATH):
@@ -50,6 +51,12 @@ _lib.int8_linear_fused_host.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64,
 _lib.int8_linear_fused_host.restype = _int
 _lib.int8_linear_fused_static.argtypes = [_vp, _i64, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i64, _int, _vp]
 _lib.int8_linear_fused_static.restype = _int
+_lib.int8_quantize_weight_per_channel_smooth.argtypes = [_vp, _i64, _i64, _i64, _vp, _vp, _vp, _vp]
+_lib.int8_quantize_weight_per_channel_smooth.restype = _int
+_lib.int8_quantize_act_per_token_smooth.argtypes = [_vp, _i64, _i64, _i64, _vp, _vp, _vp, _vp]
+_lib.int8_quantize_act_per_token_smooth.restype = _int
+_lib.int8_linear_fused_smooth.argtypes = [_vp, _i64, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i64, _vp, _sz, _vp]
+_lib.int8_linear_fused_smooth.restype = _int
 _lib.int8_gemm_i32_debug.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64, _vp, _sz, _vp]
 _lib.int8_gemm_i32_debug.restype = _int
 _lib.int8_check_status.argtypes = [_vp, _vp]
@@ -137,6 +144,58 @@ def int8_quantize_act_per_token(A: torch.Tensor, qa: torch.Tensor | None = None,
     _check(_lib.int8_quantize_act_per_token(_ptr(A), M, K, A.stride(0), _ptr(qa), _ptr(s_tok), _stream(A)),
            "int8_quantize_act_per_token")
     return qa, s_tok
+
+
+def int8_quantize_weight_per_channel_smooth(W: torch.Tensor, w_mult: torch.Tensor):
+    """fp32 [N,K] times the per-input-channel factors fp32 [K] (SmoothQuant hook) -> (int8 [N,K], fp32 [N])."""
+    _need(W, torch.float32, "W", 2)
+    _need(w_mult, torch.float32, "w_mult", 1)
+    N, K = W.shape
+    if w_mult.shape[0] != K:
+        raise ValueError("w_mult must have K entries")
+    qw = torch.empty((N, K), dtype=torch.int8, device=W.device)
+    s_ch = torch.empty((N,), dtype=torch.float32, device=W.device)
+    _check(_lib.int8_quantize_weight_per_channel_smooth(_ptr(W), N, K, W.stride(0), _ptr(w_mult), _ptr(qw), _ptr(s_ch),
+                                                        _stream(W)), "int8_quantize_weight_per_channel_smooth")
+    return qw, s_ch
+
+
+def int8_quantize_act_per_token_smooth(A: torch.Tensor, a_mult: torch.Tensor):
+    """bf16 [M,K] times the per-input-channel factors fp32 [K] (SmoothQuant hook) -> (int8 [M,K], fp32 [M])."""
+    _need(A, torch.bfloat16, "A", 2)
+    _need(a_mult, torch.float32, "a_mult", 1)
+    M, K = A.shape
+    if a_mult.shape[0] != K:
+        raise ValueError("a_mult must have K entries")
+    qa = torch.empty((M, K), dtype=torch.int8, device=A.device)
+    s_tok = torch.empty((M,), dtype=torch.float32, device=A.device)
+    _check(_lib.int8_quantize_act_per_token_smooth(_ptr(A), M, K, A.stride(0), _ptr(a_mult), _ptr(qa), _ptr(s_tok),
+                                                   _stream(A)), "int8_quantize_act_per_token_smooth")
+    return qa, s_tok
+
+
+def int8_linear_fused_smooth(A: torch.Tensor, a_mult: torch.Tensor, qw: torch.Tensor, s_ch: torch.Tensor,
+                             bias: torch.Tensor | None = None, out: torch.Tensor | None = None,
+                             workspace: torch.Tensor | None = None) -> torch.Tensor:
+    """Fused linear on bf16 activations smoothed by a_mult (weights quantized with the matching w_mult)."""
+    _need(A, torch.bfloat16, "A", 2)
+    _need(a_mult, torch.float32, "a_mult", 1)
+    _need(qw, torch.int8, "qw", 2)
+    _need(s_ch, torch.float32, "s_ch", 1)
+    M, K = A.shape
+    N = qw.shape[0]
+    if qw.shape[1] != K or s_ch.shape[0] != N or a_mult.shape[0] != K or not qw.is_contiguous():
+        raise ValueError("shape mismatch")
+    if bias is not None:
+        _need(bias, torch.float32, "bias", 1)
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=A.device)
+    if workspace is None:
+        workspace = alloc_workspace(M, N, K, ACT_BF16, A.device)
+    _check(_lib.int8_linear_fused_smooth(_ptr(A), A.stride(0), _ptr(a_mult), _ptr(qw), _ptr(s_ch), _ptr(bias), _ptr(out),
+                                         out.stride(0), M, N, K, _ptr(workspace), workspace.numel(), _stream(A)),
+           "int8_linear_fused_smooth")
+    return out
 
 
 def int8_linear_workspace_bytes(M: int, N: int, K: int, a_dtype: int = ACT_BF16) -> int:

@@ -71,26 +71,48 @@ const char* int8_linear_config_name(int config_id) {
     return tc_config_name(config_id);
 }
 
-int int8_quantize_weight_per_channel(const float* W, int64_t N, int64_t K, int64_t ldw,
-                                     int8_t* qw, float* s_ch, void* stream) {
+static int quantize_weight_impl(const float* W, int64_t N, int64_t K, int64_t ldw, const float* mult,
+                                int8_t* qw, float* s_ch, void* stream) {
     if (W == nullptr || qw == nullptr || s_ch == nullptr) return W8A8_ERR_INVALID_ARG;
     if (N <= 0 || K <= 0 || N > INT32_MAX || K > INT32_MAX || ldw < K) return W8A8_ERR_INVALID_ARG;
-    if (K % 16 != 0 || ldw % 4 != 0 || !aligned16(W) || !aligned16(qw)) return W8A8_ERR_ALIGNMENT;
+    if (K % 16 != 0 || ldw % 4 != 0 || !aligned16(W) || !aligned16(qw) || !aligned16(mult)) return W8A8_ERR_ALIGNMENT;
     if (int e = check_arch()) return e;
-    cudaError_t ce = launch_quantize_f32(W, ldw, static_cast<int>(N), static_cast<int>(K), qw, s_ch,
+    cudaError_t ce = launch_quantize_f32(W, ldw, static_cast<int>(N), static_cast<int>(K), mult, qw, s_ch,
                                          static_cast<cudaStream_t>(stream));
     return ce == cudaSuccess ? W8A8_OK : W8A8_ERR_CUDA;
 }
 
-int int8_quantize_act_per_token(const void* A_bf16, int64_t M, int64_t K, int64_t lda,
-                                int8_t* qa, float* s_tok, void* stream) {
+static int quantize_act_impl(const void* A_bf16, int64_t M, int64_t K, int64_t lda, const float* mult,
+                             int8_t* qa, float* s_tok, void* stream) {
     if (A_bf16 == nullptr || qa == nullptr || s_tok == nullptr) return W8A8_ERR_INVALID_ARG;
     if (M <= 0 || K <= 0 || M > INT32_MAX || K > INT32_MAX || lda < K) return W8A8_ERR_INVALID_ARG;
-    if (K % 16 != 0 || lda % 8 != 0 || !aligned16(A_bf16) || !aligned16(qa)) return W8A8_ERR_ALIGNMENT;
+    if (K % 16 != 0 || lda % 8 != 0 || !aligned16(A_bf16) || !aligned16(qa) || !aligned16(mult)) return W8A8_ERR_ALIGNMENT;
     if (int e = check_arch()) return e;
-    cudaError_t ce = launch_quantize_bf16(A_bf16, lda, static_cast<int>(M), static_cast<int>(K), qa, s_tok, nullptr,
+    cudaError_t ce = launch_quantize_bf16(A_bf16, lda, static_cast<int>(M), static_cast<int>(K), mult, qa, s_tok, nullptr,
                                           static_cast<cudaStream_t>(stream));
     return ce == cudaSuccess ? W8A8_OK : W8A8_ERR_CUDA;
+}
+
+int int8_quantize_weight_per_channel(const float* W, int64_t N, int64_t K, int64_t ldw,
+                                     int8_t* qw, float* s_ch, void* stream) {
+    return quantize_weight_impl(W, N, K, ldw, nullptr, qw, s_ch, stream);
+}
+
+int int8_quantize_weight_per_channel_smooth(const float* W, int64_t N, int64_t K, int64_t ldw, const float* w_mult,
+                                            int8_t* qw, float* s_ch, void* stream) {
+    if (w_mult == nullptr) return W8A8_ERR_INVALID_ARG;
+    return quantize_weight_impl(W, N, K, ldw, w_mult, qw, s_ch, stream);
+}
+
+int int8_quantize_act_per_token(const void* A_bf16, int64_t M, int64_t K, int64_t lda,
+                                int8_t* qa, float* s_tok, void* stream) {
+    return quantize_act_impl(A_bf16, M, K, lda, nullptr, qa, s_tok, stream);
+}
+
+int int8_quantize_act_per_token_smooth(const void* A_bf16, int64_t M, int64_t K, int64_t lda, const float* a_mult,
+                                       int8_t* qa, float* s_tok, void* stream) {
+    if (a_mult == nullptr) return W8A8_ERR_INVALID_ARG;
+    return quantize_act_impl(A_bf16, M, K, lda, a_mult, qa, s_tok, stream);
 }
 
 size_t int8_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int a_dtype) {
@@ -110,11 +132,12 @@ void int8_linear_workspace_offsets(int64_t M, int64_t K, size_t* s_tok_offset, s
     if (qa_offset) *qa_offset = q_off;
 }
 
-int int8_linear_fused(const void* A, int a_dtype, int64_t lda, const float* s_tok_in,
+static int fused_impl(const void* A, int a_dtype, int64_t lda, const float* s_tok_in, const float* a_mult,
                       const int8_t* qw, const float* s_ch, const float* bias,
                       void* out_bf16, int64_t ldo, int64_t M, int64_t N, int64_t K,
                       void* workspace, size_t workspace_bytes, void* stream) {
     if (A == nullptr || qw == nullptr || s_ch == nullptr || out_bf16 == nullptr) return W8A8_ERR_INVALID_ARG;
+    if (!aligned16(a_mult)) return W8A8_ERR_ALIGNMENT;
     if (a_dtype != W8A8_ACT_BF16 && a_dtype != W8A8_ACT_INT8) return W8A8_ERR_INVALID_ARG;
     if ((a_dtype == W8A8_ACT_INT8) != (s_tok_in != nullptr)) return W8A8_ERR_INVALID_ARG;
     if (int e = check_dims(M, N, K)) return e;
@@ -142,7 +165,7 @@ int int8_linear_fused(const void* A, int a_dtype, int64_t lda, const float* s_to
         int8_t* qa = reinterpret_cast<int8_t*>(ws + q_off);
         // the quantizer clears the status word; the GEMM behind it (programmatic dependent launch) sets
         // itself up while the quantizer runs and waits for it before its first read
-        if (launch_quantize_bf16(A, lda, g.M, g.K, qa, s_tok, status, st) != cudaSuccess) return W8A8_ERR_CUDA;
+        if (launch_quantize_bf16(A, lda, g.M, g.K, a_mult, qa, s_tok, status, st) != cudaSuccess) return W8A8_ERR_CUDA;
         g.qa = qa; g.lda_q = K; g.s_tok = s_tok; g.after_quantizer = true;
     } else {
         g.qa = static_cast<const int8_t*>(A); g.lda_q = lda; g.s_tok = s_tok_in; g.after_quantizer = false;
@@ -151,6 +174,23 @@ int int8_linear_fused(const void* A, int a_dtype, int64_t lda, const float* s_to
     if ((forced < 0 && M <= kSkinnyM) || forced == tc_num_configs())
         return launch_gemm_simt(g, st) == cudaSuccess ? W8A8_OK : W8A8_ERR_CUDA;
     return launch_gemm_tc(g, forced, st);
+}
+
+int int8_linear_fused(const void* A, int a_dtype, int64_t lda, const float* s_tok_in,
+                      const int8_t* qw, const float* s_ch, const float* bias,
+                      void* out_bf16, int64_t ldo, int64_t M, int64_t N, int64_t K,
+                      void* workspace, size_t workspace_bytes, void* stream) {
+    return fused_impl(A, a_dtype, lda, s_tok_in, nullptr, qw, s_ch, bias, out_bf16, ldo, M, N, K,
+                      workspace, workspace_bytes, stream);
+}
+
+int int8_linear_fused_smooth(const void* A_bf16, int64_t lda, const float* a_mult,
+                             const int8_t* qw, const float* s_ch, const float* bias,
+                             void* out_bf16, int64_t ldo, int64_t M, int64_t N, int64_t K,
+                             void* workspace, size_t workspace_bytes, void* stream) {
+    if (a_mult == nullptr) return W8A8_ERR_INVALID_ARG;
+    return fused_impl(A_bf16, W8A8_ACT_BF16, lda, nullptr, a_mult, qw, s_ch, bias, out_bf16, ldo, M, N, K,
+                      workspace, workspace_bytes, stream);
 }
 
 int int8_linear_fused_host(const void* A_host, void* d_A,

@@ -12,10 +12,12 @@ namespace w8a8 {
 constexpr int kStatusTimeout = 7;
 
 // ---- quantize.cu
-// status_to_clear: workspace status word the kernel resets (or nullptr)
-cudaError_t launch_quantize_bf16(const void* A, int64_t lda, int M, int K, int8_t* qa, float* s_tok,
+// status_to_clear: workspace status word the kernel resets (or nullptr).
+// mult: per-input-channel factors fp32 [K] multiplied into the operand first (SmoothQuant hook), or nullptr.
+cudaError_t launch_quantize_bf16(const void* A, int64_t lda, int M, int K, const float* mult, int8_t* qa, float* s_tok,
                                  int* status_to_clear, cudaStream_t st);
-cudaError_t launch_quantize_f32(const float* W, int64_t ldw, int N, int K, int8_t* qw, float* s_ch, cudaStream_t st);
+cudaError_t launch_quantize_f32(const float* W, int64_t ldw, int N, int K, const float* mult, int8_t* qw, float* s_ch,
+                                cudaStream_t st);
 
 // ---- gemm_simt.cu : CUDA-core (dp4a) path, used for skinny M and as a cross-check
 struct GemmArgs {

@@ -19,6 +19,7 @@
 #include <cuda_bf16.h>
 
 #include <mutex>
+#include <type_traits>
 
 namespace w8a8 {
 namespace {
@@ -118,6 +119,39 @@ __device__ __forceinline__ uint2 quant8(const uint4& v, const RowScale& rs, cons
     return make_uint2(quant4(f[0], f[1], f[2], f[3], rs), quant4(f[4], f[5], f[6], f[7], rs));
 }
 
+// SmoothQuant hook: x'[k] = RN(float(x[k]) * mult[k]) before everything else. 8 smoothed values of a unit.
+__device__ __forceinline__ void smooth8(const uint4& v, const float* __restrict__ mult8, float (&f)[8]) {
+    const float4 m0 = __ldg(reinterpret_cast<const float4*>(mult8));
+    const float4 m1 = __ldg(reinterpret_cast<const float4*>(mult8) + 1);
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    const float m[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        f[2 * i] = __fmul_rn(__uint_as_float(w[i] << 16), m[2 * i]);
+        f[2 * i + 1] = __fmul_rn(__uint_as_float(w[i] & 0xffff0000u), m[2 * i + 1]);
+    }
+}
+__device__ __forceinline__ float absmax8f(const float (&f)[8], float m) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) m = fmaxf(m, fabsf(f[i]));
+    return m;
+}
+__device__ __forceinline__ uint64_t quant2f(float lo, float hi, const RowScale2& r2) {
+    const uint64_t x = pack2(lo, hi);
+    const uint64_t q0 = mul2(x, r2.inv);
+    const uint64_t r0 = fma2(r2.neg_s, q0, x);
+    const uint64_t q1 = fma2(r0, r2.inv, q0);
+    const uint64_t r1 = fma2(r2.neg_s, q1, x);
+    const uint64_t q2 = fma2(r1, r2.inv, q1);
+    return add2(q2, r2.magic);
+}
+__device__ __forceinline__ uint2 quant8f(const float (&f)[8], const RowScale& rs, const RowScale2& r2) {
+    if (rs.fast)
+        return make_uint2(gather4(quant2f(f[0], f[1], r2), quant2f(f[2], f[3], r2)),
+                          gather4(quant2f(f[4], f[5], r2), quant2f(f[6], f[7], r2)));
+    return make_uint2(quant4(f[0], f[1], f[2], f[3], rs), quant4(f[4], f[5], f[6], f[7], rs));
+}
+
 // ------------------------------------------------------------------------------------------- staged kernel
 
 constexpr int SG_WARPS = 16;                         // consumer warps per CTA (one more warp produces)
@@ -131,10 +165,12 @@ __device__ __forceinline__ void bulk_load_row(uint32_t smem_dst, const void* gsr
 }
 
 // WPR consumer warps share a row (power of two <= SG_WARPS); a stage holds RPS = SG_WARPS / WPR rows.
-template <int WPR>
+// SMOOTH: multiply every element by mult[k] first (SmoothQuant hook).
+template <int WPR, bool SMOOTH>
 __global__ void __launch_bounds__(SG_THREADS, 2)
 quant_rows_staged_kernel(const __nv_bfloat16* __restrict__ x, int64_t ld, int rows, int K,
-                         int8_t* __restrict__ q, float* __restrict__ s_out, int* status, int num_stages) {
+                         int8_t* __restrict__ q, float* __restrict__ s_out, int* status, int num_stages,
+                         const float* __restrict__ mult) {
     // a dependent kernel (the GEMM) may set itself up while this one runs; it waits for this grid before reading
     grid_dep_launch_dependents();
     if (status != nullptr && blockIdx.x == 0 && threadIdx.x == 0) *status = 0;
@@ -194,12 +230,24 @@ quant_rows_staged_kernel(const __nv_bfloat16* __restrict__ x, int64_t ld, int ro
             const int row = g * RPS + slot;
             const bool live = ok && row < rows;
             const uint4* srow = reinterpret_cast<const uint4*>(base_ptr + stage * stage_bytes + slot * row_bytes);
-            __nv_bfloat162 m2 = __float2bfloat162_rn(0.f);
-            if (live) {
+            float amax = 0.f;
+            if (SMOOTH) {
+                if (live) {
+#pragma unroll 2
+                    for (int u = part * 32 + lane; u < units; u += WPR * 32) {
+                        float f[8];
+                        smooth8(srow[u], mult + u * 8, f);
+                        amax = absmax8f(f, amax);
+                    }
+                }
+            } else {
+                __nv_bfloat162 m2 = __float2bfloat162_rn(0.f);
+                if (live) {
 #pragma unroll 3
-                for (int u = part * 32 + lane; u < units; u += WPR * 32) m2 = absmax8(srow[u], m2);
+                    for (int u = part * 32 + lane; u < units; u += WPR * 32) m2 = absmax8(srow[u], m2);
+                }
+                amax = unpack_max(m2);
             }
-            float amax = unpack_max(m2);
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
             if (WPR > 1) {
@@ -215,8 +263,17 @@ quant_rows_staged_kernel(const __nv_bfloat16* __restrict__ x, int64_t ld, int ro
                 const RowScale2 r2 = make_row_scale2(rs);
                 if (part == 0 && lane == 0) s_out[row] = rs.s;
                 uint2* qrow = reinterpret_cast<uint2*>(q + static_cast<int64_t>(row) * K);
+                if (SMOOTH) {
+#pragma unroll 2
+                    for (int u = part * 32 + lane; u < units; u += WPR * 32) {
+                        float f[8];
+                        smooth8(srow[u], mult + u * 8, f);      // the same rounded products as in the first pass
+                        qrow[u] = quant8f(f, rs, r2);
+                    }
+                } else {
 #pragma unroll 3
-                for (int u = part * 32 + lane; u < units; u += WPR * 32) qrow[u] = quant8(srow[u], rs, r2);
+                    for (int u = part * 32 + lane; u < units; u += WPR * 32) qrow[u] = quant8(srow[u], rs, r2);
+                }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(empty_bar(stage));    // this warp is done with the stage
@@ -257,6 +314,25 @@ template <> struct Chunk<float> {
 #pragma unroll
         for (int i = 0; i < 4; ++i) v[i] = __ldg(q + i);
     }
+    // 16 bf16 values widened to fp32 (exact)
+    __device__ __forceinline__ void load(const __nv_bfloat16* p) {
+        const uint4* q = reinterpret_cast<const uint4*>(p);
+        const uint4 lo = __ldg(q), hi = __ldg(q + 1);
+        const uint32_t w[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            v[i] = make_float4(__uint_as_float(w[2 * i] << 16), __uint_as_float(w[2 * i] & 0xffff0000u),
+                               __uint_as_float(w[2 * i + 1] << 16), __uint_as_float(w[2 * i + 1] & 0xffff0000u));
+    }
+    // SmoothQuant hook: one rounded multiply per element by its input channel's factor
+    __device__ __forceinline__ void scale(const float* __restrict__ mult16) {
+        const float4* m = reinterpret_cast<const float4*>(mult16);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float4 f = __ldg(m + i);
+            v[i] = make_float4(__fmul_rn(v[i].x, f.x), __fmul_rn(v[i].y, f.y), __fmul_rn(v[i].z, f.z), __fmul_rn(v[i].w, f.w));
+        }
+    }
     __device__ __forceinline__ void zero() {
 #pragma unroll
         for (int i = 0; i < 4; ++i) v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -275,10 +351,16 @@ template <> struct Chunk<float> {
 
 // WPR warps per row (a power of two <= 16); a CTA works on RPC = 16 / WPR rows at a time. Rows with more
 // than WPR*32*CPL chunks stream the surplus twice (absmax pass, then quantize pass) from memory / L2.
-template <typename T, int WPR>
+// SMOOTH (SmoothQuant hook): elements are widened to fp32 and multiplied by mult[k] as they are loaded.
+template <typename T, int WPR, bool SMOOTH>
 __global__ void __launch_bounds__(WARPS * 32, 1)
 quant_rows_kernel(const T* __restrict__ x, int64_t ld, int rows, int K,
-                  int8_t* __restrict__ q, float* __restrict__ s_out, int* status) {
+                  int8_t* __restrict__ q, float* __restrict__ s_out, int* status, const float* __restrict__ mult) {
+    using C = Chunk<typename std::conditional<SMOOTH, float, T>::type>;
+    auto fetch = [&](C& c, const T* row, int chunk) {
+        c.load(row + chunk * 16);
+        if constexpr (SMOOTH) c.scale(mult + chunk * 16);
+    };
     grid_dep_launch_dependents();
     if (status != nullptr && blockIdx.x == 0 && threadIdx.x == 0) *status = 0;
 
@@ -295,19 +377,19 @@ quant_rows_kernel(const T* __restrict__ x, int64_t ld, int rows, int K,
         const int row = base + slot;
         const bool live = row < rows;
         const T* xr = x + static_cast<int64_t>(live ? row : 0) * ld;
-        Chunk<T> reg[CPL];
+        C reg[CPL];
         float amax = 0.f;
 #pragma unroll
         for (int i = 0; i < CPL; ++i) {
             const int c = c0 + i * STRIDE;
-            if (live && c < nchunks) reg[i].load(xr + c * 16); else reg[i].zero();
+            if (live && c < nchunks) fetch(reg[i], xr, c); else reg[i].zero();
         }
 #pragma unroll
         for (int i = 0; i < CPL; ++i) amax = fmaxf(amax, reg[i].absmax());
         if (live) {
             for (int c = c0 + CPL * STRIDE; c < nchunks; c += STRIDE) {   // surplus chunks (very long rows)
-                Chunk<T> t;
-                t.load(xr + c * 16);
+                C t;
+                fetch(t, xr, c);
                 amax = fmaxf(amax, t.absmax());
             }
         }
@@ -329,8 +411,8 @@ quant_rows_kernel(const T* __restrict__ x, int64_t ld, int rows, int K,
                 if (c < nchunks) *reinterpret_cast<uint4*>(qr + c * 16) = reg[i].quantize(s);
             }
             for (int c = c0 + CPL * STRIDE; c < nchunks; c += STRIDE) {
-                Chunk<T> t;
-                t.load(xr + c * 16);
+                C t;
+                fetch(t, xr, c);
                 *reinterpret_cast<uint4*>(qr + c * 16) = t.quantize(s);
             }
         }
@@ -351,29 +433,32 @@ int sm_count() {
 }
 
 template <typename T, int WPR>
-cudaError_t launch_reg(const T* x, int64_t ld, int rows, int K, int8_t* q, float* s, int* status, cudaStream_t st) {
+cudaError_t launch_reg(const T* x, int64_t ld, int rows, int K, int8_t* q, float* s, int* status, const float* mult,
+                       cudaStream_t st) {
     constexpr int RPC = WARPS / WPR;
     const int units = (rows + RPC - 1) / RPC;
     const int cap = sm_count() * 2;
     const int grid = units < cap ? units : cap;
-    quant_rows_kernel<T, WPR><<<grid, WARPS * 32, 0, st>>>(x, ld, rows, K, q, s, status);
+    if (mult != nullptr) quant_rows_kernel<T, WPR, true><<<grid, WARPS * 32, 0, st>>>(x, ld, rows, K, q, s, status, mult);
+    else quant_rows_kernel<T, WPR, false><<<grid, WARPS * 32, 0, st>>>(x, ld, rows, K, q, s, status, nullptr);
     return cudaGetLastError();
 }
 
 template <typename T>
-cudaError_t dispatch_reg(const T* x, int64_t ld, int rows, int K, int8_t* q, float* s, int* status, cudaStream_t st) {
+cudaError_t dispatch_reg(const T* x, int64_t ld, int rows, int K, int8_t* q, float* s, int* status, const float* mult,
+                         cudaStream_t st) {
     const int nchunks = K / 16;
     // fewest warps per row that keep the whole row in registers (<= CPL chunks per lane)
-    if (nchunks <= 32 * CPL)  return launch_reg<T, 1>(x, ld, rows, K, q, s, status, st);
-    if (nchunks <= 64 * CPL)  return launch_reg<T, 2>(x, ld, rows, K, q, s, status, st);
-    if (nchunks <= 128 * CPL) return launch_reg<T, 4>(x, ld, rows, K, q, s, status, st);
-    if (nchunks <= 256 * CPL) return launch_reg<T, 8>(x, ld, rows, K, q, s, status, st);
-    return launch_reg<T, 16>(x, ld, rows, K, q, s, status, st);
+    if (nchunks <= 32 * CPL)  return launch_reg<T, 1>(x, ld, rows, K, q, s, status, mult, st);
+    if (nchunks <= 64 * CPL)  return launch_reg<T, 2>(x, ld, rows, K, q, s, status, mult, st);
+    if (nchunks <= 128 * CPL) return launch_reg<T, 4>(x, ld, rows, K, q, s, status, mult, st);
+    if (nchunks <= 256 * CPL) return launch_reg<T, 8>(x, ld, rows, K, q, s, status, mult, st);
+    return launch_reg<T, 16>(x, ld, rows, K, q, s, status, mult, st);
 }
 
 template <int WPR>
 cudaError_t launch_staged(const __nv_bfloat16* x, int64_t ld, int rows, int K, int8_t* q, float* s, int* status,
-                          cudaStream_t st) {
+                          const float* mult, cudaStream_t st) {
     constexpr int RPS = SG_WARPS / WPR;
     const int stage_bytes = RPS * K * 2;
     const int groups = (rows + RPS - 1) / RPS;
@@ -388,34 +473,41 @@ cudaError_t launch_staged(const __nv_bfloat16* x, int64_t ld, int rows, int K, i
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [] {
-        attr_err = cudaFuncSetAttribute(quant_rows_staged_kernel<WPR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        attr_err = cudaFuncSetAttribute(quant_rows_staged_kernel<WPR, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         SG_SMEM_BUDGET + 1024);
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(quant_rows_staged_kernel<WPR, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            SG_SMEM_BUDGET + 1024);
     });
     if (attr_err != cudaSuccess) return attr_err;
     const int cap = ctas_per_sm * sm_count();
     const int grid = groups < cap ? groups : cap;
-    quant_rows_staged_kernel<WPR><<<grid, SG_THREADS, smem, st>>>(x, ld, rows, K, q, s, status, num_stages);
+    if (mult != nullptr)
+        quant_rows_staged_kernel<WPR, true><<<grid, SG_THREADS, smem, st>>>(x, ld, rows, K, q, s, status, num_stages, mult);
+    else
+        quant_rows_staged_kernel<WPR, false><<<grid, SG_THREADS, smem, st>>>(x, ld, rows, K, q, s, status, num_stages, nullptr);
     return cudaGetLastError();
 }
 
 } // namespace
 
-cudaError_t launch_quantize_bf16(const void* A, int64_t lda, int M, int K, int8_t* qa, float* s_tok,
+cudaError_t launch_quantize_bf16(const void* A, int64_t lda, int M, int K, const float* mult, int8_t* qa, float* s_tok,
                                  int* status_to_clear, cudaStream_t st) {
     const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(A);
     // a warp handles up to 4 KB of a row (measured best among 1-16 KB); rows of up to 64 KB (K <= 32768) go
     // through the staged kernel, longer ones through the register kernel
     const int row_bytes = K * 2;
-    if (row_bytes <= 2048)  return launch_staged<1>(x, lda, M, K, qa, s_tok, status_to_clear, st);   // 16 rows per stage
-    if (row_bytes <= 8192)  return launch_staged<2>(x, lda, M, K, qa, s_tok, status_to_clear, st);   // 8 rows per stage
-    if (row_bytes <= 16384) return launch_staged<4>(x, lda, M, K, qa, s_tok, status_to_clear, st);
-    if (row_bytes <= 32768) return launch_staged<8>(x, lda, M, K, qa, s_tok, status_to_clear, st);
-    if (row_bytes <= 65536) return launch_staged<16>(x, lda, M, K, qa, s_tok, status_to_clear, st);
-    return dispatch_reg<__nv_bfloat16>(x, lda, M, K, qa, s_tok, status_to_clear, st);
+    if (row_bytes <= 2048)  return launch_staged<1>(x, lda, M, K, qa, s_tok, status_to_clear, mult, st);   // 16 rows per stage
+    if (row_bytes <= 8192)  return launch_staged<2>(x, lda, M, K, qa, s_tok, status_to_clear, mult, st);   // 8 rows per stage
+    if (row_bytes <= 16384) return launch_staged<4>(x, lda, M, K, qa, s_tok, status_to_clear, mult, st);
+    if (row_bytes <= 32768) return launch_staged<8>(x, lda, M, K, qa, s_tok, status_to_clear, mult, st);
+    if (row_bytes <= 65536) return launch_staged<16>(x, lda, M, K, qa, s_tok, status_to_clear, mult, st);
+    return dispatch_reg<__nv_bfloat16>(x, lda, M, K, qa, s_tok, status_to_clear, mult, st);
 }
 
-cudaError_t launch_quantize_f32(const float* W, int64_t ldw, int N, int K, int8_t* qw, float* s_ch, cudaStream_t st) {
-    return dispatch_reg<float>(W, ldw, N, K, qw, s_ch, nullptr, st);
+cudaError_t launch_quantize_f32(const float* W, int64_t ldw, int N, int K, const float* mult, int8_t* qw, float* s_ch,
+                                cudaStream_t st) {
+    return dispatch_reg<float>(W, ldw, N, K, qw, s_ch, nullptr, mult, st);
 }
 
 } // namespace w8a8

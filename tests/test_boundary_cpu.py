@@ -93,6 +93,10 @@ def test_quantizers_reject_bad_arguments():
     assert lib.int8_gemm_i32_debug(P, P, P, 8, 6, 16, P, 256, None) == 2
     assert lib.int8_gemm_i32_debug(P, P, P, 8, 8, 16, P, 8, None) == 4
     assert lib.int8_check_status(None, None) == 4
+    # SmoothQuant entry points: the factor vector is required and must be 16-byte aligned
+    assert lib.int8_quantize_weight_per_channel_smooth(P, 8, 16, 16, None, P, P, None) == 1
+    assert lib.int8_quantize_act_per_token_smooth(P, 8, 16, 16, P + 4, P, P, None) == 2
+    assert lib.int8_linear_fused_smooth(P, 64, None, P, P, None, P, 64, 32, 64, 64, P, 1 << 20, None) == 1
 
 
 def test_no_device_means_a_loud_error_not_a_fallback():

@@ -138,6 +138,58 @@ def test_weight_quantizer_bit_exact(N, K):
     assert np.array_equal(qw.cpu().numpy(), qw_ref)
 
 
+# ------------------------------------------------------------------------------- SmoothQuant hook
+
+def smooth_factor(K, seed):
+    rng = np.random.default_rng(seed)
+    return (rng.random(K) * 3 + 0.1).astype(np.float32)
+
+
+@pytest.mark.parametrize("M,K", [(1, 16), (33, 2048), (300, 3072), (40, 12288), (3, 40000)])
+def test_act_quantizer_smooth_bit_exact(M, K):
+    spec = synth.LinearSpec(f"qs{M}x{K}", M, K, 8, outlier_frac=0.01 if K >= 256 else 0.0)
+    A = synth.make_activations(spec)
+    mult = smooth_factor(K, K)
+    qa_ref, s_ref = oracle.quantize_act_per_token_smooth(synth.bf16_bits(A), mult)
+    qa, s = w8.int8_quantize_act_per_token_smooth(A.to(DEV), torch.from_numpy(mult).to(DEV))
+    assert np.array_equal(s.cpu().numpy().view(np.uint32), s_ref.view(np.uint32))
+    assert np.array_equal(qa.cpu().numpy(), qa_ref)
+
+
+@pytest.mark.parametrize("N,K", [(100, 3072), (17, 12288), (3, 16400)])
+def test_weight_quantizer_smooth_bit_exact(N, K):
+    W = synth.make_weight(synth.LinearSpec(f"ws{N}x{K}", 8, K, N))
+    mult = smooth_factor(K, N)
+    qw_ref, s_ref = oracle.quantize_weight_per_channel_smooth(W.numpy(), mult)
+    qw, s = w8.int8_quantize_weight_per_channel_smooth(W.to(DEV), torch.from_numpy(mult).to(DEV))
+    assert np.array_equal(s.cpu().numpy().view(np.uint32), s_ref.view(np.uint32))
+    assert np.array_equal(qw.cpu().numpy(), qw_ref)
+
+
+def test_fused_smooth_matches_oracle():
+    spec = synth.LinearSpec("fsmooth", 1000, 1024, 1544, outlier_frac=0.02)
+    t = synth.make_linear(spec)
+    A_bits = synth.bf16_bits(t["A"])
+    W, b = t["W"].numpy(), t["bias"].numpy()
+    # alpha = 0.5 factors from the tensors themselves (calibration stands outside the path)
+    ax = np.abs(t["A"].float().numpy()).max(axis=0).astype(np.float64)
+    aw = np.abs(W).max(axis=0).astype(np.float64)
+    sm = np.sqrt(ax / aw)
+    a_mult, w_mult = (1.0 / sm).astype(np.float32), sm.astype(np.float32)
+    qw_ref, s_ch_ref = oracle.quantize_weight_per_channel_smooth(W, w_mult)
+    ref = oracle.linear_fused_bf16_smooth(A_bits, a_mult, qw_ref, s_ch_ref, b)
+    qw, s_ch = w8.int8_quantize_weight_per_channel_smooth(t["W"].to(DEV), torch.from_numpy(w_mult).to(DEV))
+    assert np.array_equal(qw.cpu().numpy(), qw_ref) and np.array_equal(s_ch.cpu().numpy(), s_ch_ref)
+    ws = w8.alloc_workspace(spec.M, spec.N, spec.K, w8.ACT_BF16, DEV)
+    out = w8.int8_linear_fused_smooth(t["A"].to(DEV), torch.from_numpy(a_mult).to(DEV), qw, s_ch, t["bias"].to(DEV),
+                                      workspace=ws)
+    check_status(ws)
+    s_off, q_off = w8.int8_linear_workspace_offsets(spec.M, spec.K)
+    qa = ws[q_off:q_off + spec.M * spec.K].view(torch.int8).view(spec.M, spec.K).cpu().numpy()
+    assert np.array_equal(qa, ref["qa"])
+    assert_bf16_close(synth.bf16_bits(out.cpu()), ref["out"])
+
+
 # ------------------------------------------------------------------------------- raw accumulators (T2)
 
 ACC_SHAPES = [
