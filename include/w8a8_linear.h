@@ -45,7 +45,7 @@ typedef enum w8a8_status {
     W8A8_ERR_INVALID_ARG = 1, /* NULL pointer, M/N/K <= 0, ld smaller than the row, unknown dtype */
     W8A8_ERR_ALIGNMENT = 2,   /* pointer not 16-byte aligned, or K/N/ld break the 16-byte rules below */
     W8A8_ERR_K_OVERFLOW = 3,  /* K > 133144: K * 127^2 would not fit in int32 */
-    W8A8_ERR_WORKSPACE = 4,   /* workspace NULL or smaller than int8_linear_workspace_bytes() */
+    W8A8_ERR_WORKSPACE = 4,   /* workspace NULL, misaligned or smaller than int8_linear_workspace_min_bytes() */
     W8A8_ERR_ARCH = 5,        /* current device is not compute capability 10.x */
     W8A8_ERR_CUDA = 6,        /* a CUDA runtime/driver call failed (launch, descriptor encode) */
     W8A8_ERR_TIMEOUT = 7      /* a bounded device-side wait expired (reported by int8_check_status) */
@@ -80,14 +80,24 @@ int int8_quantize_act_per_token(const void* A_bf16, int64_t M, int64_t K, int64_
                                 int8_t* qa, float* s_tok, void* stream);
 
 /*
- * Bytes of caller-provided device workspace int8_linear_fused needs for this
+ * Bytes of caller-provided device workspace to give int8_linear_fused for this
  * problem (0 on invalid sizes). Layout, from the workspace base (which must be
  * 256-byte aligned): a 256-byte status block; then, for bf16 activations only,
- * s_tok as fp32 [M] (padded to 256 bytes) and qa as int8 [M,K] dense. The
- * workspace needs no initialisation. After a bf16 call the caller may read qa
- * and s_tok back from there (int8_linear_workspace_offsets gives the offsets).
+ * s_tok as fp32 [M] (padded to 256 bytes) and qa as int8 [M,K] dense; then, for
+ * shapes whose last wave of output tiles is mostly empty, room for int32 partial
+ * accumulators (the tiles of that wave are cut along K over the idle SMs and
+ * summed exactly; at most about 10 MB). The workspace needs no initialisation.
+ * After a bf16 call the caller may read qa and s_tok back from there
+ * (int8_linear_workspace_offsets gives the offsets).
  */
 size_t int8_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int a_dtype);
+
+/*
+ * The smallest workspace int8_linear_fused accepts: the layout above without the
+ * partial accumulators. With less than int8_linear_workspace_bytes() the results
+ * are the same bit for bit; shapes with a mostly empty last wave run slower.
+ */
+size_t int8_linear_workspace_min_bytes(int64_t M, int64_t N, int64_t K, int a_dtype);
 
 /* Byte offsets of s_tok and qa inside the workspace for bf16 activations. */
 void int8_linear_workspace_offsets(int64_t M, int64_t K, size_t* s_tok_offset, size_t* qa_offset);
@@ -105,8 +115,9 @@ void int8_linear_workspace_offsets(int64_t M, int64_t K, size_t* s_tok_offset, s
  *   s_ch      in   fp32 [N]
  *   bias      in   fp32 [N] or NULL (no bias term)
  *   out_bf16  out  bf16 [M,N], row stride ldo elements (multiple of 8), 16-byte aligned
- *   workspace      device scratch of at least int8_linear_workspace_bytes(); two calls that
- *                  may overlap on the device need distinct workspaces
+ *   workspace      device scratch, int8_linear_workspace_bytes() for full speed and at least
+ *                  int8_linear_workspace_min_bytes(); two calls that may overlap on the device
+ *                  need distinct workspaces
  * Requires K % 16 == 0, N % 8 == 0, K <= W8A8_K_MAX. The kernel configuration
  * (tile shape, pipeline depth, skinny-M path) is chosen from (M,N,K); the
  * paper's per-shape autotuning ("Why autotuning is load-bearing") is replaced
@@ -167,7 +178,7 @@ int int8_linear_fused_host(const void* A_host, void* d_A,
  *                   W8A8_ERR_TIMEOUT if a bounded device-side wait gave up (as int8_check_status does).
  *
  * Limits and rules:
- *   - Problems whose scratch, int8_linear_workspace_bytes(M, N, K, W8A8_ACT_BF16), exceeds
+ *   - Problems whose scratch, int8_linear_workspace_min_bytes(M, N, K, W8A8_ACT_BF16), exceeds
  *     W8A8_STATIC_WORKSPACE_BYTES are refused with W8A8_ERR_WORKSPACE before anything is enqueued
  *     (roughly M * (K + 4) <= 16 MiB: e.g. M = 4608 tokens at K = 3072, not at K = 12288).
  *   - The first call on each device looks up the array's device address (a one-time set-up step under a
@@ -188,7 +199,8 @@ int int8_linear_fused_static(const void* A_bf16, int64_t lda,
  * Test-only export of the raw accumulators of the tensor-core path (the int32
  * values the fused epilogue consumes): acc[m,n] = sum_k qa[m,k] * qw[n,k].
  *   qa in int8 [M,K] dense; qw in int8 [N,K] dense; acc out int32 [M,N] dense (N % 4 == 0);
- *   workspace as for int8_linear_fused with W8A8_ACT_INT8.
+ *   workspace as for int8_linear_fused with W8A8_ACT_INT8 (256 bytes at least; given
+ *   int8_linear_workspace_bytes() it also takes the K-split path of the fused call).
  */
 int int8_gemm_i32_debug(const int8_t* qa, const int8_t* qw, int32_t* acc,
                         int64_t M, int64_t N, int64_t K,
@@ -202,8 +214,21 @@ int int8_gemm_i32_debug(const int8_t* qa, const int8_t* qw, int32_t* acc,
  */
 int int8_check_status(void* workspace, void* stream);
 
-/* Force a kernel configuration for sweeps (-1 = choose from the shape). Returns the previous value. */
+/*
+ * Force a kernel configuration for sweeps and tests. -1 = choose from the shape; -2 = choose from the shape
+ * but never cut tiles along K; id = that configuration; id + 0x100 = that configuration, never cut along K.
+ * Returns the previous value.
+ */
 int int8_linear_force_config(int config_id);
+
+/*
+ * Reports how int8_linear_fused would run this problem on the current device with a workspace of
+ * workspace_bytes (under the forced configuration, if one is set): the kernel configuration, the number
+ * of CTAs or CTA pairs launched, and the K-split of the last wave (split_tiles tiles cut into split_parts
+ * parts each; both 0 when nothing is cut). Any output pointer may be NULL. Launches nothing.
+ */
+int int8_linear_plan(int64_t M, int64_t N, int64_t K, int a_dtype, size_t workspace_bytes,
+                     int* config_id, int* cta_groups, int* split_tiles, int* split_parts);
 
 /* Number of kernel configurations, and a short description of one (NULL if out of range). */
 int int8_linear_num_configs(void);

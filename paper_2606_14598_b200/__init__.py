@@ -9,5 +9,5 @@ from .binding import (  # noqa: F401
     int8_gemm_i32_debug, int8_linear_fused, int8_linear_fused_host, int8_linear_fused_static, int8_linear_workspace_bytes,
     int8_linear_workspace_offsets, int8_quantize_act_per_token, int8_quantize_weight_per_channel, num_configs,
     int8_quantize_act_per_token_smooth, int8_quantize_weight_per_channel_smooth, int8_linear_fused_smooth,
-    status_string,
+    status_string, int8_linear_workspace_min_bytes, int8_linear_plan,
 )

@@ -26,7 +26,7 @@ EXPORTS = (
     "int8_linear_workspace_offsets", "int8_linear_fused", "int8_linear_fused_host", "int8_gemm_i32_debug",
     "int8_check_status", "int8_linear_force_config", "int8_linear_num_configs", "int8_linear_config_name",
     "int8_status_string", "int8_linear_fused_static", "int8_quantize_weight_per_channel_smooth",
-    "int8_quantize_act_per_token_smooth", "int8_linear_fused_smooth",
+    "int8_quantize_act_per_token_smooth", "int8_linear_fused_smooth", "int8_linear_workspace_min_bytes", "int8_linear_plan",
 )
 
 if not os.path.exists(LIB_PATH):
@@ -43,6 +43,10 @@ _lib.int8_quantize_act_per_token.argtypes = [_vp, _i64, _i64, _i64, _vp, _vp, _v
 _lib.int8_quantize_act_per_token.restype = _int
 _lib.int8_linear_workspace_bytes.argtypes = [_i64, _i64, _i64, _int]
 _lib.int8_linear_workspace_bytes.restype = _sz
+_lib.int8_linear_workspace_min_bytes.argtypes = [_i64, _i64, _i64, _int]
+_lib.int8_linear_workspace_min_bytes.restype = _sz
+_lib.int8_linear_plan.argtypes = [_i64, _i64, _i64, _int, _sz] + [ctypes.POINTER(_int)] * 4
+_lib.int8_linear_plan.restype = _int
 _lib.int8_linear_workspace_offsets.argtypes = [_i64, _i64, ctypes.POINTER(_sz), ctypes.POINTER(_sz)]
 _lib.int8_linear_workspace_offsets.restype = None
 _lib.int8_linear_fused.argtypes = [_vp, _int, _i64, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i64, _vp, _sz, _vp]
@@ -200,6 +204,21 @@ def int8_linear_fused_smooth(A: torch.Tensor, a_mult: torch.Tensor, qw: torch.Te
 
 def int8_linear_workspace_bytes(M: int, N: int, K: int, a_dtype: int = ACT_BF16) -> int:
     return int(_lib.int8_linear_workspace_bytes(M, N, K, a_dtype))
+
+
+def int8_linear_workspace_min_bytes(M: int, N: int, K: int, a_dtype: int = ACT_BF16) -> int:
+    return int(_lib.int8_linear_workspace_min_bytes(M, N, K, a_dtype))
+
+
+def int8_linear_plan(M: int, N: int, K: int, a_dtype: int = ACT_BF16, workspace_bytes: int | None = None) -> dict:
+    """How the fused call would run this shape: {'config', 'name', 'groups', 'split_tiles', 'split_parts'}."""
+    if workspace_bytes is None:
+        workspace_bytes = int8_linear_workspace_bytes(M, N, K, a_dtype)
+    v = [_int(0) for _ in range(4)]
+    _check(_lib.int8_linear_plan(M, N, K, a_dtype, workspace_bytes, *[ctypes.byref(x) for x in v]), "int8_linear_plan")
+    cfg = int(v[0].value)
+    return {"config": cfg, "name": config_name(cfg), "groups": int(v[1].value),
+            "split_tiles": int(v[2].value), "split_parts": int(v[3].value)}
 
 
 def int8_linear_workspace_offsets(M: int, K: int):

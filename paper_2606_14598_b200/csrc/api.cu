@@ -115,13 +115,41 @@ int int8_quantize_act_per_token_smooth(const void* A_bf16, int64_t M, int64_t K,
     return quantize_act_impl(A_bf16, M, K, lda, a_mult, qa, s_tok, stream);
 }
 
-size_t int8_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int a_dtype) {
+size_t int8_linear_workspace_min_bytes(int64_t M, int64_t N, int64_t K, int a_dtype) {
     if (M <= 0 || N <= 0 || K <= 0) return 0;
     if (a_dtype == W8A8_ACT_INT8) return kStatusBlock;
     if (a_dtype != W8A8_ACT_BF16) return 0;
     size_t s_off, q_off;
     offsets(M, &s_off, &q_off);
     return q_off + round_up(static_cast<size_t>(M) * static_cast<size_t>(K), 256);
+}
+
+size_t int8_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int a_dtype) {
+    const size_t base = int8_linear_workspace_min_bytes(M, N, K, a_dtype);
+    if (base == 0 || M <= kSkinnyM || M > INT32_MAX || N > INT32_MAX || K > W8A8_K_MAX) return base;
+    // room for the partial accumulators of the K-split, where the automatic choice would use one
+    return base + round_up(tc_max_scratch_bytes(static_cast<int>(M), static_cast<int>(N), static_cast<int>(K)), 256);
+}
+
+int int8_linear_plan(int64_t M, int64_t N, int64_t K, int a_dtype, size_t workspace_bytes,
+                     int* config_id, int* cta_groups, int* split_tiles, int* split_parts) {
+    if (int e = check_dims(M, N, K)) return e;
+    const size_t base = int8_linear_workspace_min_bytes(M, N, K, a_dtype);
+    if (base == 0) return W8A8_ERR_INVALID_ARG;
+    if (workspace_bytes < base) return W8A8_ERR_WORKSPACE;
+    if (int e = check_arch()) return e;          // the plan depends on the device's SM count
+    const int forced = g_forced_config.load();
+    TcPlan plan{};
+    if ((forced < 0 && M <= kSkinnyM) || (forced >= 0 && (forced & 0xff) == tc_num_configs())) {
+        plan.config = tc_num_configs();
+    } else {
+        plan = tc_plan(static_cast<int>(M), static_cast<int>(N), static_cast<int>(K), forced, workspace_bytes - base);
+    }
+    if (config_id) *config_id = plan.config;
+    if (cta_groups) *cta_groups = plan.groups;
+    if (split_tiles) *split_tiles = plan.split_tiles;
+    if (split_parts) *split_parts = plan.split_parts;
+    return W8A8_OK;
 }
 
 void int8_linear_workspace_offsets(int64_t M, int64_t K, size_t* s_tok_offset, size_t* qa_offset) {
@@ -146,18 +174,29 @@ static int fused_impl(const void* A, int a_dtype, int64_t lda, const float* s_to
     if (N % 8 != 0 || ldo % 8 != 0 || lda_bytes % 16 != 0) return W8A8_ERR_ALIGNMENT;
     if (!aligned16(A) || !aligned16(qw) || !aligned16(out_bf16)) return W8A8_ERR_ALIGNMENT;
     if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0 ||
-        workspace_bytes < int8_linear_workspace_bytes(M, N, K, a_dtype))
+        workspace_bytes < int8_linear_workspace_min_bytes(M, N, K, a_dtype))
         return W8A8_ERR_WORKSPACE;
     if (int e = check_arch()) return e;
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     int* status = reinterpret_cast<int*>(ws);
+    const int forced = g_forced_config.load();
+    const bool simt = (forced < 0 && M <= kSkinnyM) || (forced >= 0 && (forced & 0xff) == tc_num_configs());
+    // whatever the workspace holds beyond the required part is scratch for the K-split of the partial wave
+    const size_t scratch_off = int8_linear_workspace_min_bytes(M, N, K, a_dtype);
+    TcPlan plan{};
+    if (!simt) {
+        plan = tc_plan(static_cast<int>(M), static_cast<int>(N), static_cast<int>(K), forced, workspace_bytes - scratch_off);
+        // arrival counters and partial sums start at zero (ahead of the quantizer, so the GEMM still launches right behind it)
+        if (plan.split_parts >= 2 && cudaMemsetAsync(ws + scratch_off, 0, plan.scratch_bytes, st) != cudaSuccess)
+            return W8A8_ERR_CUDA;
+    }
 
     GemmArgs g{};
     g.qw = qw; g.s_ch = s_ch; g.bias = bias; g.out = out_bf16; g.ldo = ldo;
     g.M = static_cast<int>(M); g.N = static_cast<int>(N); g.K = static_cast<int>(K);
-    g.raw_i32 = false; g.status = status;
+    g.raw_i32 = false; g.status = status; g.split_ws = plan.split_parts >= 2 ? ws + scratch_off : nullptr;
     if (a_dtype == W8A8_ACT_BF16) {
         size_t s_off, q_off;
         offsets(M, &s_off, &q_off);
@@ -170,10 +209,8 @@ static int fused_impl(const void* A, int a_dtype, int64_t lda, const float* s_to
     } else {
         g.qa = static_cast<const int8_t*>(A); g.lda_q = lda; g.s_tok = s_tok_in; g.after_quantizer = false;
     }
-    const int forced = g_forced_config.load();
-    if ((forced < 0 && M <= kSkinnyM) || forced == tc_num_configs())
-        return launch_gemm_simt(g, st) == cudaSuccess ? W8A8_OK : W8A8_ERR_CUDA;
-    return launch_gemm_tc(g, forced, st);
+    if (simt) return launch_gemm_simt(g, st) == cudaSuccess ? W8A8_OK : W8A8_ERR_CUDA;
+    return launch_gemm_tc(g, plan, st);
 }
 
 int int8_linear_fused(const void* A, int a_dtype, int64_t lda, const float* s_tok_in,
@@ -225,11 +262,17 @@ int int8_gemm_i32_debug(const int8_t* qa, const int8_t* qw, int32_t* acc,
     GemmArgs g{};
     g.qa = qa; g.lda_q = K; g.s_tok = nullptr; g.qw = qw; g.s_ch = nullptr; g.bias = nullptr;
     g.out = acc; g.ldo = N; g.M = static_cast<int>(M); g.N = static_cast<int>(N); g.K = static_cast<int>(K);
-    g.raw_i32 = true; g.status = status; g.after_quantizer = false;
+    g.raw_i32 = true; g.status = status; g.after_quantizer = false; g.split_ws = nullptr;
     const int forced = g_forced_config.load();
-    if ((forced < 0 && M <= kSkinnyM) || forced == tc_num_configs())
+    if ((forced < 0 && M <= kSkinnyM) || (forced >= 0 && (forced & 0xff) == tc_num_configs()))
         return launch_gemm_simt(g, st) == cudaSuccess ? W8A8_OK : W8A8_ERR_CUDA;
-    return launch_gemm_tc(g, forced, st);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    const TcPlan plan = tc_plan(g.M, g.N, g.K, forced, workspace_bytes - kStatusBlock);
+    if (plan.split_parts >= 2) {
+        if (cudaMemsetAsync(ws + kStatusBlock, 0, plan.scratch_bytes, st) != cudaSuccess) return W8A8_ERR_CUDA;
+        g.split_ws = ws + kStatusBlock;
+    }
+    return launch_gemm_tc(g, plan, st);
 }
 
 int int8_check_status(void* workspace, void* stream) {

@@ -23,6 +23,13 @@
 // Two accumulators of BN columns alternate in TMEM so that the epilogue of one
 // tile overlaps the k-loop of the next.
 //
+// K-split of the partial wave: when the number of tiles is not a multiple of the number of CTA groups, the
+// last num_tiles % groups tiles would keep only a few SMs busy for a whole tile time. The host may ask for
+// them to be cut along K into split_s parts, one part per group. Every part adds its int32 partial
+// accumulator into the tile's slab of the workspace (integer sums: the result does not depend on the
+// order); a per-tile counter tells the part that finishes last to read the sums back and run the epilogue.
+// No CTA ever waits for another one.
+//
 // Every mbarrier wait is bounded: on expiry the CTA records W8A8_ERR_TIMEOUT in
 // the workspace status word, all roles unwind, TMEM is freed and the kernel
 // returns.
@@ -66,7 +73,8 @@ struct SmemLayout {
     static constexpr int NUM_BARS = NUM_FULL + STAGES + 4;
     static constexpr int OFF_TMEM = OFF_BARS + NUM_BARS * 8;
     static constexpr int OFF_ABORT = OFF_TMEM + 4;
-    static constexpr int TOTAL = OFF_ABORT + 4;
+    static constexpr int OFF_LAST = OFF_ABORT + 4;                 // "this CTA finishes the split tile" (epilogue warps)
+    static constexpr int TOTAL = OFF_LAST + 4;
     static constexpr int DYN_BYTES = TOTAL + 1024;                 // slack to align the base to 1024
 };
 
@@ -80,7 +88,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                const __grid_constant__ CUtensorMap tm_out,
                const float* __restrict__ s_tok, const float* __restrict__ s_ch, const float* __restrict__ bias,
-               int32_t* __restrict__ raw_out, int M, int N, int K, int* status, int after_quantizer, int raster_gn) {
+               int32_t* __restrict__ raw_out, int M, int N, int K, int* status, int after_quantizer, int raster_gn,
+               int split_tiles, int split_s, int32_t* split_slabs, int* split_counters) {
     using L = SmemLayout<CG, BN, STAGES, KBS>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -100,7 +109,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::OFF_ABORT);
     const WaitCtl ctl{abort_flag, status, WAIT_LIMIT_NS};
 
-    constexpr uint32_t TMEM_COLS = 2 * BN;      // 512 or 256: a power of two >= 32
+    // two accumulators, each at a power-of-two column offset (the allocation must be a power of two >= 32)
+    constexpr uint32_t TMEM_BUF = BN <= 128 ? 128u : 256u;
+    constexpr uint32_t TMEM_COLS = 2 * TMEM_BUF;
+    static_assert(BN % 64 == 0 && BN <= 256, "BN: whole 64-column output boxes, at most 256 TMEM columns per buffer");
 
     // without a quantizer ahead of it (which clears the status word) the kernel clears it itself; a time-out
     // can only be recorded seconds later
@@ -132,6 +144,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     const int num_tiles = num_m * num_n;
     const int num_kb = (K + BK - 1) / BK;
     const int first_tile = blockIdx.x / CG, tile_step = gridDim.x / CG;
+    // Work list of this CTA group: whole tiles first_tile, first_tile + tile_step, ... below tiles_whole, then
+    // (K-split) part unit_part of tile unit_tile: stages [unit_sb, unit_se) of its k-loop.
+    const int num_kstages = (num_kb + KBS - 1) / KBS;
+    const int tiles_whole = num_tiles - split_tiles;
+    const bool has_unit = split_s >= 2 && first_tile < split_tiles * split_s;
+    const int unit_slot = has_unit ? first_tile / split_s : 0, unit_part = has_unit ? first_tile % split_s : 0;
+    const int unit_tile = tiles_whole + unit_slot;
+    const int unit_sb = has_unit ? num_kstages * unit_part / split_s : 0;
+    const int unit_se = has_unit ? num_kstages * (unit_part + 1) / split_s : 0;
     // Tile order: bands of raster_gn tile columns; inside a band the column index runs fastest, then the
     // row block. raster_gn = 1 walks along M first, raster_gn >= num_n along N first. A wave of concurrent
     // tiles then covers about (wave / gn) row blocks x gn columns: A and W lines are shared by a balanced
@@ -156,12 +177,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         uint32_t phase = 0;
         int issued = 0;
         bool ok = true;
-        for (int t = first_tile; t < num_tiles && ok; t += tile_step) {
+        auto produce = [&](int t, int sb, int se) {
             const int m0 = tile_m(t) * TILE_M + rank * BM;
             const int n0 = tile_n(t) * BN + rank * L::B_ROWS;
             if (lane == 0) {
                 const uint64_t keep = l2_policy_evict_last();        // operands are re-read by other tiles: keep them in L2
-                for (int kb = 0; kb < num_kb; kb += KBS) {
+                for (int ks = sb; ks < se; ++ks) {
+                    const int kb = ks * KBS;
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, ctl, W_PRODUCER_EMPTY, kStatusTimeout)) { ok = false; break; }
                     // a stage always receives all its k-blocks: those past the end of K are zero-filled by TMA
                     // (and skipped by the MMA thread), which keeps the byte count of the barrier constant
@@ -185,7 +207,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 }
             }
             ok = __all_sync(0xffffffffu, ok) != 0;
-        }
+        };
+        for (int t = first_tile; t < tiles_whole && ok; t += tile_step) produce(t, 0, num_kstages);
+        if (has_unit && ok) produce(unit_tile, unit_sb, unit_se);
         if (!ok && lane == 0 && (CG == 1 || leader)) {
             // let copies that are still in flight land before the CTA goes away
             int s = stage;
@@ -205,12 +229,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             uint32_t phase = 0;
             bool ok = true;
             int it = 0;
-            for (int t = first_tile; t < num_tiles && ok; t += tile_step, ++it) {
+            auto mma_tile = [&](int sb, int se) {
                 const int buf = it & 1;
-                if (!mbar_wait(tempty_bar(buf), ((it >> 1) & 1) ^ 1u, ctl, W_MMA_TMEM_EMPTY, kStatusTimeout)) { ok = false; break; }
+                if (!mbar_wait(tempty_bar(buf), ((it >> 1) & 1) ^ 1u, ctl, W_MMA_TMEM_EMPTY, kStatusTimeout)) { ok = false; return; }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + buf * BN;
-                for (int kb = 0; kb < num_kb; kb += KBS) {
+                const uint32_t d_tmem = tmem_base + buf * TMEM_BUF;
+                for (int ks = sb; ks < se; ++ks) {
+                    const int kb = ks * KBS;
 #pragma unroll
                     for (int sub = 0; sub < KBS; ++sub) {
                         if (!mbar_wait(full_bar(stage, sub), phase, ctl, W_MMA_FULL, kStatusTimeout)) { ok = false; break; }
@@ -224,7 +249,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 #pragma unroll
                         for (int k = 0; k < BK / MMA_K; ++k) {
                             if (k < ksteps) {   // advancing K by 32 bytes inside the swizzled row: +2 in 16-byte units
-                                const uint32_t acc = (kb | sub | k) != 0 ? 1u : 0u;
+                                const uint32_t acc = ((ks - sb) | sub | k) != 0 ? 1u : 0u;   // the first MMA overwrites
                                 if (CG == 2) mma_i8_ss_pair(d_tmem, da + 2 * k, db + 2 * k, idesc, acc);
                                 else mma_i8_ss(d_tmem, da + 2 * k, db + 2 * k, idesc, acc);
                             }
@@ -241,7 +266,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     if (CG == 2) { tc_commit_pair(tfull_bar(buf)); tc_commit_pair(mapa_shared(tfull_bar(buf), 1)); }
                     else tc_commit(tfull_bar(buf));
                 }
-            }
+            };
+            for (int t = first_tile; t < tiles_whole && ok; t += tile_step, ++it) mma_tile(0, num_kstages);
+            if (has_unit && ok) mma_tile(unit_sb, unit_se);
         }
     } else {
         // ------------------------------------------------------------ epilogue (warps 2..5)
@@ -256,7 +283,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         if (after_quantizer) grid_dep_wait();          // s_tok comes from the kernel before this one
         bool ok = true;
         int it = 0;
-        for (int t = first_tile; t < num_tiles; t += tile_step, ++it) {
+        volatile int* last_flag = reinterpret_cast<volatile int*>(base_ptr + L::OFF_LAST);
+        auto epi_tile = [&](int t, bool unit) {
             const int buf = it & 1;
             const int m0 = tile_m(t) * TILE_M + rank * BM, n0 = tile_n(t) * BN;
             if (!RAW_I32) {
@@ -272,9 +300,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             const float st = (!RAW_I32 && row < M) ? __ldg(s_tok + row) : 0.f;
             if (ok && !mbar_wait(tfull_bar(buf), (it >> 1) & 1, ctl, W_EPI_TMEM_FULL, kStatusTimeout)) ok = false;
             ok = __all_sync(0xffffffffu, ok);
-            if (!ok) continue;                         // keep taking the named barriers, skip the work
+            if (!ok && !unit) return;                  // later tiles still take their named barriers, but skip the work
             tc_fence_after();
-            const uint32_t t_row = tmem_base + (static_cast<uint32_t>(lg * 32) << 16) + buf * BN;
+            const uint32_t t_row = tmem_base + (static_cast<uint32_t>(lg * 32) << 16) + buf * TMEM_BUF;
             // One chunk = 32 accumulator columns of this thread's row. Two chunks make a 32 x 64 output box.
             // The TMEM load of the next chunk is in flight while the current one is converted.
             const uint64_t st2 = pack2(st, st);
@@ -339,18 +367,67 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             };
             constexpr int CHUNKS = BN / 32;
             uint32_t va[32], vb[32];
-            tmem_ld_32x32b_x32(t_row, va);
+            if (!unit) {
+                tmem_ld_32x32b_x32(t_row, va);
 #pragma unroll 1
-            for (int cc = 0; cc < CHUNKS; cc += 2) {
-                tmem_wait_ld();
-                tmem_ld_32x32b_x32(t_row + (cc + 1) * 32, vb);
-                process(cc, va);
-                tmem_wait_ld();
-                if (cc + 2 < CHUNKS) tmem_ld_32x32b_x32(t_row + (cc + 2) * 32, va);
-                else release_accumulator();
-                process(cc + 1, vb);
+                for (int cc = 0; cc < CHUNKS; cc += 2) {
+                    tmem_wait_ld();
+                    tmem_ld_32x32b_x32(t_row + (cc + 1) * 32, vb);
+                    process(cc, va);
+                    tmem_wait_ld();
+                    if (cc + 2 < CHUNKS) tmem_ld_32x32b_x32(t_row + (cc + 2) * 32, va);
+                    else release_accumulator();
+                    process(cc + 1, vb);
+                }
+                return;
             }
-        }
+            // ---- one K part of a split tile. Every part adds its int32 accumulators into the tile's slab in
+            // global memory (zeroed by the host before the launch) with reductions, which need no reply. Slab
+            // layout: [CTA of the pair][column][128 rows], so that the 32 rows of a warp are 128 contiguous bytes.
+            constexpr int SLAB = BN * BM;
+            int32_t* slab = split_slabs + static_cast<size_t>(unit_slot * CG + rank) * SLAB;
+            if (ok) {
+                int32_t* mine = slab + lg * 32 + lane;
+                auto put = [&](int cc, const uint32_t (&v)[32]) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) red_add_s32(mine + (cc * 32 + j) * BM, static_cast<int32_t>(v[j]));
+                };
+                tmem_ld_32x32b_x32(t_row, va);
+#pragma unroll 1
+                for (int cc = 0; cc < CHUNKS; cc += 2) {
+                    tmem_wait_ld();
+                    tmem_ld_32x32b_x32(t_row + (cc + 1) * 32, vb);
+                    put(cc, va);
+                    tmem_wait_ld();
+                    if (cc + 2 < CHUNKS) tmem_ld_32x32b_x32(t_row + (cc + 2) * 32, va);
+                    else release_accumulator();
+                    put(cc + 1, vb);
+                }
+            }
+            // The part that arrives last at the tile's counter finishes the tile (fence, then count: every
+            // reduction counted before ours has been applied before we read the slab).
+            __threadfence();
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (ep_tid == 0) *last_flag = atomicAdd(split_counters + unit_slot * CG + rank, 1) == split_s - 1 ? 1 : 0;
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (*last_flag == 0 || !ok) return;
+            __threadfence();
+            // This is the CTA's last piece of work and its MMAs have completed: the operand ring is free. Pull the
+            // whole slab into it with asynchronous copies (all in flight at once), then run the usual epilogue.
+            static_assert(SLAB * 4 <= STAGES * L::STAGE_BYTES, "the slab fits in the operand ring");
+            for (int i = ep_tid; i < SLAB / 4; i += EPI_THREADS) cp_async_16(base + i * 16, slab + i * 4);
+            cp_async_wait_all();
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            const int32_t* sm_slab = reinterpret_cast<const int32_t*>(base_ptr) + lg * 32 + lane;
+#pragma unroll 1
+            for (int cc = 0; cc < CHUNKS; ++cc) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) va[j] = static_cast<uint32_t>(sm_slab[(cc * 32 + j) * BM]);
+                process(cc, va);
+            }
+        };
+        for (int t = first_tile; t < tiles_whole; t += tile_step, ++it) epi_tile(t, false);
+        if (has_unit) epi_tile(unit_tile, true);
         if (!RAW_I32 && lane == 0) bulk_wait_group<0>();
     }
 
@@ -398,16 +475,22 @@ bool encode_2d(CUtensorMap* tm, CUtensorMapDataType dt, const void* ptr, uint64_
 struct TcConfig {
     const char* name;
     int cg, bn, stages, kbs;
+    float eff;      // measured throughput per SM relative to configuration 2 (large shapes, whole waves)
 };
 constexpr TcConfig kConfigs[] = {
-    // measured on the c4 shapes (hot L2): pair 3 x 256 B: 117 / 111 us; pair 5 x 128 B: 125 / 120 us;
-    // pair 2 x 384 B: 127 / 131 us; one CTA 4 x 128 B: 131 / 124 us; one CTA 2 x 256 B: 144 / 136 us
-    {"tc 128x256 per CTA, 4 stages x 128 B of K", 1, 256, 4, 1},
-    {"tc 128x128 per CTA, 3 stages x 256 B of K", 1, 128, 3, 2},
-    {"tc 256x256 per CTA pair, 3 stages x 256 B of K", 2, 256, 3, 2},
-    {"tc 256x128 per CTA pair, 4 stages x 256 B of K", 2, 128, 4, 2},
+    // measured on the c4 shapes (hot L2): pair 256x256 3 x 256 B: 115 / 111 us; one CTA 128x256 4 x 128 B: 129 / 121 us;
+    // pair 256x192: 130 / 123 us; one CTA 128x128: 164 / 154 us; pair 256x128: 168 / 162 us
+    {"tc 128x256 per CTA, 4 stages x 128 B of K", 1, 256, 4, 1, 0.89f},
+    {"tc 128x128 per CTA, 3 stages x 256 B of K", 1, 128, 3, 2, 0.72f},
+    {"tc 256x256 per CTA pair, 3 stages x 256 B of K", 2, 256, 3, 2, 1.00f},
+    {"tc 256x128 per CTA pair, 4 stages x 256 B of K", 2, 128, 4, 2, 0.70f},
+    {"tc 256x192 per CTA pair, 3 stages x 256 B of K", 2, 192, 3, 2, 0.88f},
 };
 constexpr int kNumConfigs = sizeof(kConfigs) / sizeof(kConfigs[0]);
+constexpr int kNoSplitBit = 0x100;        // added to a forced configuration id: no K-split of the partial wave
+constexpr size_t kCounterBytes = 1024;    // per-tile arrival counters at the head of the split scratch (<= 148 ints)
+constexpr int kMaxSplit = 8;              // parts per tile
+constexpr int kMinStagesPerPart = 4;
 
 int sm_count() {
     static int n = [] {
@@ -424,7 +507,7 @@ int sm_count() {
 int raster_band(const GemmArgs&) { return 1 << 20; }
 
 template <int CG, int BN, int STAGES, int KBS, bool RAW>
-int launch_cfg(const GemmArgs& a, cudaStream_t st) {
+int launch_cfg(const GemmArgs& a, const TcPlan& plan, cudaStream_t st) {
     using L = SmemLayout<CG, BN, STAGES, KBS>;
     static_assert(L::DYN_BYTES <= 232448, "shared memory budget");
     auto kern = gemm_tc_kernel<CG, BN, STAGES, KBS, RAW>;
@@ -441,10 +524,8 @@ int launch_cfg(const GemmArgs& a, cudaStream_t st) {
     } else {
         if (!encode_2d(&tm_out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, a.out, a.M, a.N, a.ldo * 2, 32, 64)) return 6;
     }
-    const int num_tiles = ((a.M + BM * CG - 1) / (BM * CG)) * ((a.N + BN - 1) / BN);
-    const int max_groups = sm_count() / CG;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(CG * (num_tiles < max_groups ? num_tiles : max_groups));
+    cfg.gridDim = dim3(CG * plan.groups);
     cfg.blockDim = dim3(NUM_THREADS);
     cfg.dynamicSmemBytes = L::DYN_BYTES;
     cfg.stream = st;
@@ -466,32 +547,71 @@ int launch_cfg(const GemmArgs& a, cudaStream_t st) {
     cfg.numAttrs = na;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tm_a, tm_b, tm_out, a.s_tok, a.s_ch, a.bias,
                                        RAW ? static_cast<int32_t*>(a.out) : nullptr, a.M, a.N, a.K, a.status,
-                                       a.after_quantizer ? 1 : 0, raster_band(a));
+                                       a.after_quantizer ? 1 : 0, raster_band(a), plan.split_tiles, plan.split_parts,
+                                       reinterpret_cast<int32_t*>(static_cast<uint8_t*>(a.split_ws) + kCounterBytes),
+                                       static_cast<int*>(a.split_ws));
     return e == cudaSuccess ? 0 : 6;
 }
 
 template <bool RAW>
-int launch_by_id(int id, const GemmArgs& a, cudaStream_t st) {
-    switch (id) {
-        case 0: return launch_cfg<1, 256, 4, 1, RAW>(a, st);
-        case 1: return launch_cfg<1, 128, 3, 2, RAW>(a, st);
-        case 2: return launch_cfg<2, 256, 3, 2, RAW>(a, st);
-        case 3: return launch_cfg<2, 128, 4, 2, RAW>(a, st);
+int launch_by_id(const GemmArgs& a, const TcPlan& plan, cudaStream_t st) {
+    switch (plan.config) {
+        case 0: return launch_cfg<1, 256, 4, 1, RAW>(a, plan, st);
+        case 1: return launch_cfg<1, 128, 3, 2, RAW>(a, plan, st);
+        case 2: return launch_cfg<2, 256, 3, 2, RAW>(a, plan, st);
+        case 3: return launch_cfg<2, 128, 4, 2, RAW>(a, plan, st);
+        case 4: return launch_cfg<2, 192, 3, 2, RAW>(a, plan, st);
         default: return 1;
     }
 }
 
-int pick_config(int M, int N, int K) {
-    (void)K;
-    // From measurements on the five benchmark shapes: CTA pairs win once there are about two waves of
-    // 256x256 pair tiles; below that one CTA per 128x256 tile fills the SMs better; tiny problems take
-    // 128x128 tiles.
-    const long n256 = (N + 255) / 256;
-    const long pair_tiles = static_cast<long>((M + 2 * BM - 1) / (2 * BM)) * n256;
-    const long tiles256 = static_cast<long>((M + BM - 1) / BM) * n256;
-    if (pair_tiles >= 2 * (sm_count() / 2)) return 2;
-    if (tiles256 >= sm_count()) return 0;
-    return 1;
+// Grid and K-split of one configuration on one shape, with its estimated run time in microseconds.
+// Whole waves of tiles cost a tile time each; the partial wave (tiles % groups, or all tiles when there are
+// fewer tiles than groups) is cut along K into as many parts as there are idle groups (at least
+// kMinStagesPerPart pipeline stages per part, at most kMaxSplit parts, and only if the scratch has room),
+// which shortens it to 1/parts of a tile time plus the cost of adding the partial sums up. With only_if_faster
+// the cut is dropped when the estimate says it does not pay (it pays for deep K: K >= ~8192).
+TcPlan plan_config(int id, int M, int N, int K, bool allow_split, bool only_if_faster, size_t scratch_bytes, double* est_us) {
+    const TcConfig& c = kConfigs[id];
+    TcPlan p{};
+    p.config = id;
+    const int max_groups = sm_count() / c.cg;
+    const long tiles = static_cast<long>((M + BM * c.cg - 1) / (BM * c.cg)) * ((N + c.bn - 1) / c.bn);
+    const int whole_waves = static_cast<int>(tiles / max_groups);
+    const int rest = static_cast<int>(tiles % max_groups);
+    const int kstages = ((K + BK - 1) / BK + c.kbs - 1) / c.kbs;
+    int parts = 1;
+    if (allow_split && rest > 0) {
+        parts = max_groups / rest;
+        if (parts > kstages / kMinStagesPerPart) parts = kstages / kMinStagesPerPart;
+        if (parts > kMaxSplit) parts = kMaxSplit;
+        const size_t need = kCounterBytes + static_cast<size_t>(rest) * c.cg * c.bn * BM * sizeof(int32_t);
+        if (parts < 2 || need > scratch_bytes) parts = 1;
+    }
+    // ~20.3 int8 TOPS per SM for configuration 2 in whole waves. A partial wave that is left whole runs its
+    // tiles faster than that (measured ~0.72 of the tile time with few SMs active: the operand traffic of a full
+    // wave is what holds the rate down); a wave cut along K keeps every SM busy and pays ~10 us for zeroing the
+    // slabs, the reductions, the pipeline refill and the read-back.
+    const double tile_us = 2.0 * BM * c.bn * static_cast<double>(K) / 20.3e6 / c.eff;
+    const double fixed_us = 4.0;                       // launch, pipeline fill, last epilogue
+    const double whole_rest_us = tile_us * (0.72 + 0.28 * rest / max_groups);
+    const double split_rest_us = tile_us / parts + 10.0;
+    if (parts > 1 && only_if_faster && split_rest_us >= whole_rest_us) parts = 1;
+    double est = fixed_us + whole_waves * tile_us;
+    if (rest > 0) est += parts > 1 ? split_rest_us : whole_rest_us;
+    if (parts > 1) {
+        p.split_tiles = rest;
+        p.split_parts = parts;
+        p.groups = whole_waves > 0 ? max_groups : rest * parts;
+        p.scratch_bytes = kCounterBytes + static_cast<size_t>(rest) * c.cg * c.bn * BM * sizeof(int32_t);
+    } else {
+        p.split_tiles = 0;
+        p.split_parts = 0;
+        p.groups = static_cast<int>(tiles < max_groups ? tiles : max_groups);
+        p.scratch_bytes = 0;
+    }
+    if (est_us) *est_us = est;
+    return p;
 }
 
 } // namespace
@@ -499,9 +619,31 @@ int pick_config(int M, int N, int K) {
 int tc_num_configs() { return kNumConfigs; }
 const char* tc_config_name(int id) { return (id >= 0 && id < kNumConfigs) ? kConfigs[id].name : nullptr; }
 
-int launch_gemm_tc(const GemmArgs& a, int forced, cudaStream_t st) {
-    const int id = (forced >= 0 && forced < kNumConfigs) ? forced : pick_config(a.M, a.N, a.K);
-    return a.raw_i32 ? launch_by_id<true>(id, a, st) : launch_by_id<false>(id, a, st);
+TcPlan tc_plan(int M, int N, int K, int forced, size_t scratch_bytes) {
+    // forced: -1 automatic, -2 automatic without K-split, id, or id + 0x100 for that configuration without K-split
+    const bool allow_split = forced == -1 || (forced >= 0 && (forced & kNoSplitBit) == 0);
+    const int id = forced < 0 ? -1 : (forced & (kNoSplitBit - 1));
+    if (id >= 0 && id < kNumConfigs) return plan_config(id, M, N, K, allow_split, false, scratch_bytes, nullptr);   // forced: cut whenever possible
+    // lowest estimated time; on (near) ties the earlier entry of this preference order wins
+    const int order[kNumConfigs] = {2, 0, 4, 3, 1};
+    TcPlan best{};
+    double best_us = 0.0;
+    for (int i = 0; i < kNumConfigs; ++i) {
+        double us = 0.0;
+        const TcPlan p = plan_config(order[i], M, N, K, allow_split, true, scratch_bytes, &us);
+        if (i == 0 || us < best_us * 0.97) { best = p; best_us = us; }
+    }
+    return best;
+}
+
+size_t tc_max_scratch_bytes(int M, int N, int K) {
+    // what the automatic choice would use with unlimited scratch
+    return tc_plan(M, N, K, -1, static_cast<size_t>(-1)).scratch_bytes;
+}
+
+int launch_gemm_tc(const GemmArgs& a, const TcPlan& plan, cudaStream_t st) {
+    if (plan.split_parts >= 2 && a.split_ws == nullptr) return 1;
+    return a.raw_i32 ? launch_by_id<true>(a, plan, st) : launch_by_id<false>(a, plan, st);
 }
 
 } // namespace w8a8

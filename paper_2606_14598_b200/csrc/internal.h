@@ -33,13 +33,27 @@ struct GemmArgs {
     bool raw_i32;
     int* status;           // workspace status word
     bool after_quantizer;  // launched behind the quantizer with programmatic dependent launch
+    void* split_ws;        // scratch of the K-split (counters, then partial accumulators), or nullptr
 };
 cudaError_t launch_gemm_simt(const GemmArgs& a, cudaStream_t st);
 
 // ---- gemm_tc.cu : tcgen05 path
 int tc_num_configs();
 const char* tc_config_name(int id);
-// Picks a configuration for the shape (or `forced` if >= 0) and launches. Returns a w8a8_status.
-int launch_gemm_tc(const GemmArgs& a, int forced, cudaStream_t st);
+// How a shape is run: configuration, grid, and the K-split of the partial wave of tiles (0 parts = none).
+struct TcPlan {
+    int config;
+    int groups;            // CTAs (or CTA pairs) launched
+    int split_tiles;       // tiles of the partial wave that are cut along K
+    int split_parts;       // parts per such tile
+    size_t scratch_bytes;  // scratch the split needs (counters, then one int32 slab per tile); all zero at launch
+};
+// Picks a configuration for the shape (or `forced` if >= 0; forced + 0x100 = that configuration without K-split).
+// A split is planned only if its scratch fits in scratch_bytes.
+TcPlan tc_plan(int M, int N, int K, int forced, size_t scratch_bytes);
+// Scratch the automatic choice uses when it is given enough.
+size_t tc_max_scratch_bytes(int M, int N, int K);
+// Launches the plan. Returns a w8a8_status.
+int launch_gemm_tc(const GemmArgs& a, const TcPlan& plan, cudaStream_t st);
 
 } // namespace w8a8

@@ -46,7 +46,7 @@ extern "C" int int8_linear_fused_static(const void* A_bf16, int64_t lda,
                                         void* out_bf16, int64_t ldo, int64_t M, int64_t N, int64_t K,
                                         int sync_and_check, void* stream) {
     // size check first: it needs no device and gives the caller a clear answer
-    const size_t need = int8_linear_workspace_bytes(M, N, K, W8A8_ACT_BF16);
+    const size_t need = int8_linear_workspace_min_bytes(M, N, K, W8A8_ACT_BF16);
     if (need == 0) return W8A8_ERR_INVALID_ARG;
     if (need > kStaticWorkspaceBytes) return W8A8_ERR_WORKSPACE;
 

@@ -347,6 +347,73 @@ def test_run_to_run_identical_and_host_buffer_entry_point():
     assert torch.equal(out_host, first.cpu())
 
 
+# ------------------------------------------------------------------------------- K-split of the partial wave
+
+# (M, N, K, configuration): shapes whose last (or only) wave of tiles leaves SMs idle, so that its tiles
+# are cut along K and the int32 partial sums are added up by the part that finishes last
+SPLIT_SHAPES = [
+    (256, 512, 2048, 2),      # two pair tiles, two parts each
+    (300, 520, 2064, 2),      # ragged M, N and K
+    (256, 256, 8192, 2),      # one tile in eight parts
+    (130, 264, 4096, 0),      # one CTA per tile
+    (300, 400, 4096, 4),      # 192-column tiles
+    (512, 5120, 2048, 3),     # 80 pair tiles on 74 pairs: a whole wave, then 6 tiles in parts
+    (512, 4864, 2048, 1),     # 152 tiles on 148 CTAs
+]
+
+
+@pytest.mark.parametrize("M,N,K,cfg", SPLIT_SHAPES)
+def test_k_split_accumulators_and_outputs_bit_exact(M, N, K, cfg):
+    rng = np.random.default_rng(M + 3 * N + 5 * K + cfg)
+    qa, qw = rand_codes(rng, (M, K)), rand_codes(rng, (N, K))
+    s_tok = (rng.random(M) * 0.05 + 0.01).astype(np.float32)
+    s_ch = (rng.random(N) * 0.0008 + 0.0002).astype(np.float32)
+    bias = (rng.standard_normal(N) * 0.01).astype(np.float32)
+    ref = oracle.linear_fused_int8(qa, s_tok, qw, s_ch, bias)
+    dev = [torch.from_numpy(a).to(DEV) for a in (qa, qw, s_tok, s_ch, bias)]
+    ws = w8.alloc_workspace(M, N, K, w8.ACT_INT8, DEV)
+    ws_big = torch.empty(ws.numel() + (32 << 20), dtype=torch.uint8, device=DEV)   # room for any split
+    for forced, want_split in ((cfg, True), (cfg + 0x100, False)):
+        w8.force_config(forced)
+        plan = w8.int8_linear_plan(M, N, K, w8.ACT_INT8, ws_big.numel())
+        assert plan["config"] == cfg and (plan["split_parts"] >= 2) == want_split, plan
+        ws_big.fill_(0x5A)                              # the scratch needs no initialisation
+        acc = w8.int8_gemm_i32_debug(dev[0], dev[1], ws_big)
+        check_status(ws_big)
+        assert np.array_equal(acc.cpu().numpy(), ref["acc"]), plan
+        for _ in range(2):                              # twice on the same scratch
+            out = w8.int8_linear_fused(dev[0], dev[1], dev[3], dev[4], s_tok=dev[2], workspace=ws_big)
+            check_status(ws_big)
+            assert_bf16_close(synth.bf16_bits(out.cpu()), ref["out"])
+    # a workspace of the minimum size turns the split off and gives the same output
+    w8.force_config(cfg)
+    ws_min = torch.empty(w8.int8_linear_workspace_min_bytes(M, N, K, w8.ACT_INT8), dtype=torch.uint8, device=DEV)
+    assert w8.int8_linear_plan(M, N, K, w8.ACT_INT8, ws_min.numel())["split_parts"] == 0
+    out = w8.int8_linear_fused(dev[0], dev[1], dev[3], dev[4], s_tok=dev[2], workspace=ws_min)
+    check_status(ws_min)
+    assert_bf16_close(synth.bf16_bits(out.cpu()), ref["out"])
+
+
+def test_k_split_from_bf16_automatic_choice():
+    # few tiles and a deep K: the automatic choice cuts along K (when the workspace has the room it asks for)
+    spec = synth.LinearSpec("split_bf16", 500, 8192, 776)
+    t = synth.make_linear(spec)
+    qw_ref, s_ch_ref = oracle.quantize_weight_per_channel(t["W"].numpy())
+    ref = oracle.linear_fused_bf16(synth.bf16_bits(t["A"]), qw_ref, s_ch_ref, t["bias"].numpy())
+    qw, s_ch = w8.int8_quantize_weight_per_channel(t["W"].to(DEV))
+    ws = w8.alloc_workspace(spec.M, spec.N, spec.K, w8.ACT_BF16, DEV)
+    assert ws.numel() > w8.int8_linear_workspace_min_bytes(spec.M, spec.N, spec.K, w8.ACT_BF16)
+    assert w8.int8_linear_plan(spec.M, spec.N, spec.K, w8.ACT_BF16, ws.numel())["split_parts"] >= 2
+    out = w8.int8_linear_fused(t["A"].to(DEV), qw, s_ch, t["bias"].to(DEV), workspace=ws)
+    check_status(ws)
+    assert_bf16_close(synth.bf16_bits(out.cpu()), ref["out"])
+    w8.force_config(-2)                                 # same shape, never cut
+    assert w8.int8_linear_plan(spec.M, spec.N, spec.K, w8.ACT_BF16, ws.numel())["split_parts"] == 0
+    out2 = w8.int8_linear_fused(t["A"].to(DEV), qw, s_ch, t["bias"].to(DEV), workspace=ws)
+    check_status(ws)
+    assert torch.equal(out, out2)
+
+
 # ------------------------------------------------------------------------------- benchmark configs, full size (T4)
 
 def sample_rows(M, n=48):
