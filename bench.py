@@ -345,7 +345,10 @@ def main():
             tg = batch_time(gemm_only)
             tq = batch_time(quant_only)
             tf_ = batch_time(fused)
+            plan = w8.int8_linear_plan(M, N, K, w8.ACT_BF16, rot[0]["ws"].numel())
             per_shape.append({"name": spec.name, "M": M, "K": K, "N": N,
+                              "kernel_config": plan["name"], "cta_groups": plan["groups"],
+                              "k_split": f"{plan['split_tiles']} tiles x {plan['split_parts']} parts" if plan["split_parts"] else "none",
                               "fused_from_bf16_us": tf_ * 1e6, "fused_from_bf16_tops": spec.ops / tf_ / 1e12,
                               "pct_of_int8_peak": 100.0 * spec.ops / tf_ / 1e12 / INT8_PEAK_TOPS,
                               "gemm_epilogue_us": tg * 1e6, "gemm_epilogue_tops": spec.ops / tg / 1e12,
@@ -403,6 +406,30 @@ def main():
                            "h2d_bytes_per_step": sum(2 * s.M * s.K for s in specs),
                            "d2h_bytes_per_step": sum(2 * s.M * s.N for s in specs), "ms_per_step": e2e_sec * 1e3,
                            "entry": "int8_linear_fused_host (pinned host bf16 in, pinned host bf16 out)"}
+
+            # ---- the same step replayed from CUDA graphs (one per rotating set): no per-call host work
+            graphs = []
+            for i in range(len(step_args)):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g):
+                    gs = torch.cuda.current_stream(dev).cuda_stream
+                    for a_ in step_args[i]:
+                        raw.int8_linear_fused(*(a_[:-1] + (gs,)))
+                graphs.append(g)
+            n_g = max(50, min(args.steps, 500))
+            for i in range(5):
+                graphs[i % len(graphs)].replay()
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for i in range(n_g):
+                graphs[i % len(graphs)].replay()
+            b.record()
+            torch.cuda.synchronize()
+            g_sec = a.elapsed_time(b) * 1e-3 / n_g
+            line["graph_replay"] = {"value": ops_per_step / g_sec / 1e12, "unit": "TOPS", "ms_per_step": g_sec * 1e3,
+                                    "steps": n_g, "note": "one captured CUDA graph per rotating input set"}
+            del graphs
 
             # ---- context on the same box: library bf16 matmul and library int8 matmul on the same shapes
             ctx = []

@@ -414,6 +414,45 @@ def test_k_split_from_bf16_automatic_choice():
     assert torch.equal(out, out2)
 
 
+# ------------------------------------------------------------------------------- CUDA graph of a block's linears
+
+def test_cuda_graph_replay_of_several_linears():
+    # the calls allocate nothing and only enqueue work on the caller's stream, so a set of linears can be
+    # captured once and replayed on new activations written into the same buffers
+    shapes = [(300, 384, 328), (300, 320, 1024), (256, 8192, 264), (2, 384, 512)]   # plain, chained sizes, K-split, skinny
+    layers = []
+    for i, (M, K, N) in enumerate(shapes):
+        spec = synth.LinearSpec(f"graph{i}", M, K, N)
+        t = synth.make_linear(spec)
+        qw_ref, s_ch_ref = oracle.quantize_weight_per_channel(t["W"].numpy())
+        qw, s_ch = w8.int8_quantize_weight_per_channel(t["W"].to(DEV))
+        layers.append({"spec": spec, "qw_ref": qw_ref, "s_ch_ref": s_ch_ref, "bias_np": t["bias"].numpy(),
+                       "A": t["A"].to(DEV), "qw": qw, "s_ch": s_ch, "bias": t["bias"].to(DEV),
+                       "out": torch.empty((M, N), dtype=torch.bfloat16, device=DEV),
+                       "ws": w8.alloc_workspace(M, N, K, w8.ACT_BF16, DEV)})
+
+    def run_all():
+        for L in layers:
+            w8.int8_linear_fused(L["A"], L["qw"], L["s_ch"], L["bias"], out=L["out"], workspace=L["ws"])
+
+    run_all()                                           # first calls (one-time set-up) outside the capture
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        run_all()
+    for seed in (11, 12):
+        for L in layers:
+            L["A_new"] = synth.make_activations(L["spec"], seed)
+            L["A"].copy_(L["A_new"].to(DEV))
+            L["out"].fill_(-3.0)
+        graph.replay()
+        torch.cuda.synchronize()
+        for L in layers:
+            check_status(L["ws"])
+            ref = oracle.linear_fused_bf16(synth.bf16_bits(L["A_new"]), L["qw_ref"], L["s_ch_ref"], L["bias_np"])
+            assert_bf16_close(synth.bf16_bits(L["out"].cpu()), ref["out"])
+
+
 # ------------------------------------------------------------------------------- benchmark configs, full size (T4)
 
 def sample_rows(M, n=48):
