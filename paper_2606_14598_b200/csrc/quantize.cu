@@ -157,6 +157,7 @@ __device__ __forceinline__ uint2 quant8f(const float (&f)[8], const RowScale& rs
 constexpr int SG_WARPS = 16;                         // consumer warps per CTA (one more warp produces)
 constexpr int SG_THREADS = (SG_WARPS + 1) * 32;
 constexpr int SG_SMEM_BUDGET = 200 * 1024;           // shared memory for the rings of one SM
+constexpr int SG_SMEM_MAX = 226 * 1024;              // all a CTA can have: only for rows too long for the budget above
 constexpr uint64_t SG_WAIT_LIMIT_NS = 2000000000ull; // bounded waits, as everywhere
 
 __device__ __forceinline__ void bulk_load_row(uint32_t smem_dst, const void* gsrc, uint32_t bytes, uint32_t bar) {
@@ -467,6 +468,8 @@ cudaError_t launch_staged(const __nv_bfloat16* x, int64_t ld, int rows, int K, i
     const int ctas_per_sm = (groups >= 8 * sm_count() && SG_SMEM_BUDGET / 2 >= 2 * stage_bytes) ? 2 : 1;
     int num_stages = SG_SMEM_BUDGET / ctas_per_sm / stage_bytes;
     if (num_stages > 8) num_stages = 8;
+    // very long rows (one row per stage, 64-113 KB): two stages out of everything a CTA can have
+    if (num_stages < 2 && 2 * stage_bytes + 1024 <= SG_SMEM_MAX) num_stages = 2;
     // the ring indices of the kernel wrap at num_stages: a ring of fewer than two stages must never be launched
     if (num_stages < 2) return cudaErrorInvalidConfiguration;
     const int smem = num_stages * stage_bytes + 16 * num_stages + SG_WARPS * 4 + 16 + 128;
@@ -474,10 +477,10 @@ cudaError_t launch_staged(const __nv_bfloat16* x, int64_t ld, int rows, int K, i
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [] {
         attr_err = cudaFuncSetAttribute(quant_rows_staged_kernel<WPR, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        SG_SMEM_BUDGET + 1024);
+                                        SG_SMEM_MAX);
         if (attr_err == cudaSuccess)
             attr_err = cudaFuncSetAttribute(quant_rows_staged_kernel<WPR, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            SG_SMEM_BUDGET + 1024);
+                                            SG_SMEM_MAX);
     });
     if (attr_err != cudaSuccess) return attr_err;
     const int cap = ctas_per_sm * sm_count();
@@ -495,13 +498,14 @@ cudaError_t launch_quantize_bf16(const void* A, int64_t lda, int M, int K, const
                                  int* status_to_clear, cudaStream_t st) {
     const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(A);
     // a warp handles up to 4 KB of a row (measured best among 1-16 KB); rows of up to 64 KB (K <= 32768) go
-    // through the staged kernel, longer ones through the register kernel
+    // through the staged kernel with several stages, rows of up to 113 KB with two stages of one row each (a warp
+    // then walks up to 7 KB), longer ones through the register kernel
     const int row_bytes = K * 2;
     if (row_bytes <= 2048)  return launch_staged<1>(x, lda, M, K, qa, s_tok, status_to_clear, mult, st);   // 16 rows per stage
     if (row_bytes <= 8192)  return launch_staged<2>(x, lda, M, K, qa, s_tok, status_to_clear, mult, st);   // 8 rows per stage
     if (row_bytes <= 16384) return launch_staged<4>(x, lda, M, K, qa, s_tok, status_to_clear, mult, st);
     if (row_bytes <= 32768) return launch_staged<8>(x, lda, M, K, qa, s_tok, status_to_clear, mult, st);
-    if (row_bytes <= 65536) return launch_staged<16>(x, lda, M, K, qa, s_tok, status_to_clear, mult, st);
+    if (2 * row_bytes + 1024 <= SG_SMEM_MAX) return launch_staged<16>(x, lda, M, K, qa, s_tok, status_to_clear, mult, st);
     return dispatch_reg<__nv_bfloat16>(x, lda, M, K, qa, s_tok, status_to_clear, mult, st);
 }
 

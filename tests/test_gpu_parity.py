@@ -67,7 +67,8 @@ def rand_codes(rng, shape, lo=-127):
 # ------------------------------------------------------------------------------- quantizers (T1)
 
 @pytest.mark.parametrize("M,K", [(1, 16), (7, 48), (33, 2048), (300, 3072), (9, 4096), (5, 8192), (40, 12288),
-                                 (3, 16384), (3, 16400), (2, 40000)])
+                                 (3, 16384), (3, 16400), (2, 40000), (150, 53248), (3, 57600), (3, 57616),
+                                 (2, 66000), (2, 133136)])
 def test_act_quantizer_bit_exact(M, K):
     spec = synth.LinearSpec(f"q{M}x{K}", M, K, 8, outlier_frac=0.01 if K >= 256 else 0.0)
     A = synth.make_activations(spec)
@@ -145,7 +146,7 @@ def smooth_factor(K, seed):
     return (rng.random(K) * 3 + 0.1).astype(np.float32)
 
 
-@pytest.mark.parametrize("M,K", [(1, 16), (33, 2048), (300, 3072), (40, 12288), (3, 40000)])
+@pytest.mark.parametrize("M,K", [(1, 16), (33, 2048), (300, 3072), (40, 12288), (3, 40000), (150, 53248), (2, 66000)])
 def test_act_quantizer_smooth_bit_exact(M, K):
     spec = synth.LinearSpec(f"qs{M}x{K}", M, K, 8, outlier_frac=0.01 if K >= 256 else 0.0)
     A = synth.make_activations(spec)
