@@ -26,6 +26,7 @@ __global__ void __launch_bounds__(WARPS * 32)
 gemm_simt_kernel(const int8_t* __restrict__ qa, int64_t lda_q, const float* __restrict__ s_tok,
                  const int8_t* __restrict__ qw, const float* __restrict__ s_ch, const float* __restrict__ bias,
                  void* __restrict__ out, int64_t ldo, int M, int N, int K, int raw_i32, int after_quantizer, int* status) {
+    grid_dep_launch_dependents();      // a following kernel launched to allow it may set itself up early
     // no quantizer ahead of this kernel to clear the status word: do it here (this kernel has no waits that could set it)
     if (!after_quantizer && status != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *status = 0;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;

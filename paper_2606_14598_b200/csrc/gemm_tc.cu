@@ -91,6 +91,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                int32_t* __restrict__ raw_out, int M, int N, int K, int* status, int after_quantizer, int raster_gn,
                int split_tiles, int split_s, int32_t* split_slabs, int* split_counters) {
     using L = SmemLayout<CG, BN, STAGES, KBS>;
+    // the next kernel in the stream, if it was launched to allow it (the next call's quantizer is), may be scheduled
+    // as this grid's CTAs retire and set itself up; it waits for this whole grid before it touches global memory
+    grid_dep_launch_dependents();
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));

@@ -174,7 +174,6 @@ quant_rows_staged_kernel(const __nv_bfloat16* __restrict__ x, int64_t ld, int ro
                          const float* __restrict__ mult) {
     // a dependent kernel (the GEMM) may set itself up while this one runs; it waits for this grid before reading
     grid_dep_launch_dependents();
-    if (status != nullptr && blockIdx.x == 0 && threadIdx.x == 0) *status = 0;
 
     constexpr int RPS = SG_WARPS / WPR;
     extern __shared__ uint8_t smem_raw[];
@@ -199,6 +198,10 @@ quant_rows_staged_kernel(const __nv_bfloat16* __restrict__ x, int64_t ld, int ro
         fence_mbar_init();
     }
     __syncthreads();
+    // This kernel may itself have been launched early, behind a kernel that allowed it (programmatic dependent
+    // launch): everything above touched shared memory only; global memory is touched after that kernel is complete.
+    grid_dep_wait();
+    if (status != nullptr && blockIdx.x == 0 && threadIdx.x == 0) *status = 0;
 
     const int total_groups = (rows + RPS - 1) / RPS;          // a group = the rows of one stage
 
@@ -363,6 +366,7 @@ quant_rows_kernel(const T* __restrict__ x, int64_t ld, int rows, int K,
         if constexpr (SMOOTH) c.scale(mult + chunk * 16);
     };
     grid_dep_launch_dependents();
+    grid_dep_wait();                      // launched early behind a kernel that allowed it: wait for that kernel's results
     if (status != nullptr && blockIdx.x == 0 && threadIdx.x == 0) *status = 0;
 
     constexpr int RPC = WARPS / WPR;
@@ -423,6 +427,23 @@ quant_rows_kernel(const T* __restrict__ x, int64_t ld, int rows, int K,
 
 // ------------------------------------------------------------------------------------------- host side
 
+// Launch that may start while the kernel ahead of it in the stream is still finishing (if that kernel allows it);
+// the kernels above wait for it with griddepcontrol.wait before they touch global memory.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kern)(KArgs...), int grid, int block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 int sm_count() {
     static int n = [] {
         int dev = 0, v = 0;
@@ -440,9 +461,9 @@ cudaError_t launch_reg(const T* x, int64_t ld, int rows, int K, int8_t* q, float
     const int units = (rows + RPC - 1) / RPC;
     const int cap = sm_count() * 2;
     const int grid = units < cap ? units : cap;
-    if (mult != nullptr) quant_rows_kernel<T, WPR, true><<<grid, WARPS * 32, 0, st>>>(x, ld, rows, K, q, s, status, mult);
-    else quant_rows_kernel<T, WPR, false><<<grid, WARPS * 32, 0, st>>>(x, ld, rows, K, q, s, status, nullptr);
-    return cudaGetLastError();
+    const float* no_mult = nullptr;
+    if (mult != nullptr) return launch_pdl(quant_rows_kernel<T, WPR, true>, grid, WARPS * 32, 0, st, x, ld, rows, K, q, s, status, mult);
+    return launch_pdl(quant_rows_kernel<T, WPR, false>, grid, WARPS * 32, 0, st, x, ld, rows, K, q, s, status, no_mult);
 }
 
 template <typename T>
@@ -485,11 +506,10 @@ cudaError_t launch_staged(const __nv_bfloat16* x, int64_t ld, int rows, int K, i
     if (attr_err != cudaSuccess) return attr_err;
     const int cap = ctas_per_sm * sm_count();
     const int grid = groups < cap ? groups : cap;
+    const float* no_mult = nullptr;
     if (mult != nullptr)
-        quant_rows_staged_kernel<WPR, true><<<grid, SG_THREADS, smem, st>>>(x, ld, rows, K, q, s, status, num_stages, mult);
-    else
-        quant_rows_staged_kernel<WPR, false><<<grid, SG_THREADS, smem, st>>>(x, ld, rows, K, q, s, status, num_stages, nullptr);
-    return cudaGetLastError();
+        return launch_pdl(quant_rows_staged_kernel<WPR, true>, grid, SG_THREADS, smem, st, x, ld, rows, K, q, s, status, num_stages, mult);
+    return launch_pdl(quant_rows_staged_kernel<WPR, false>, grid, SG_THREADS, smem, st, x, ld, rows, K, q, s, status, num_stages, no_mult);
 }
 
 } // namespace
