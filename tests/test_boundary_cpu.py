@@ -44,6 +44,18 @@ def test_workspace_sizes():
     assert s_off == 256 and q_off == 512 and w8.int8_linear_workspace_bytes(2, 8, 3072, w8.ACT_BF16) == 512 + 6144
     assert w8.int8_linear_workspace_bytes(0, 8, 16) == 0
     assert w8.int8_linear_workspace_bytes(8, 8, 16, 5) == 0
+    # the smallest accepted workspace is the layout above; the recommended one adds room for the partial sums of
+    # the K-split where the shape's last wave of tiles is mostly empty and K is deep (the paper's llm-proj), and
+    # nothing where it is not (the c4 shapes) or where the CUDA-core path runs (M <= 16)
+    for (M, N, K) in [(4608, 3072, 12288), (4608, 12288, 3072), (4110, 4608, 53248), (512, 4608, 53248), (2, 18432, 3072)]:
+        for dt in (w8.ACT_BF16, w8.ACT_INT8):
+            lo, hi = w8.int8_linear_workspace_min_bytes(M, N, K, dt), w8.int8_linear_workspace_bytes(M, N, K, dt)
+            assert lo % 256 == 0 and hi % 256 == 0 and lo <= hi <= lo + (12 << 20)
+            if dt == w8.ACT_BF16:
+                assert lo == w8.int8_linear_workspace_offsets(M, K)[1] + (M * K + 255) // 256 * 256
+            else:
+                assert lo == 256
+            assert (hi > lo) == (K == 53248), (M, N, K, lo, hi)
 
 
 def test_configs_are_listed():
@@ -77,7 +89,7 @@ def test_fused_rejects_bad_arguments_before_any_launch():
     assert fused(a_dtype=1, s_tok=P, lda=72) == ALIGN       # int8 row stride not a multiple of 16 bytes
     assert fused(A=P + 8) == ALIGN and fused(qw=P + 4) == ALIGN and fused(out=P + 2) == ALIGN
     assert fused(ws=None) == WS and fused(ws=P + 128) == WS and fused(ws_bytes=255) == WS
-    need = w8.int8_linear_workspace_bytes(32, 64, 64, 0)
+    need = w8.int8_linear_workspace_min_bytes(32, 64, 64, 0)
     assert fused(ws_bytes=need - 1) == WS
 
 
