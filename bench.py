@@ -301,6 +301,12 @@ def main():
         "pct_of_int8_peak": 100.0 * tops / (INT8_PEAK_TOPS * world), "int8_peak_tops": INT8_PEAK_TOPS,
         "clocks": clocks.summary(), "gpu_launches": launches,
     }
+    # what the tensor pipes could do at the clock seen: 16384 int8 ops per clock per SM (8192 multiply-adds)
+    if line["clocks"]["sm_mhz"]:
+        sms = torch.cuda.get_device_properties(dev).multi_processor_count
+        ceiling = sms * 16384 * line["clocks"]["sm_mhz"] * 1e6 / 1e12
+        line["int8_ceiling_at_observed_clock"] = {"tops": ceiling, "sm_mhz": line["clocks"]["sm_mhz"], "sms": sms,
+                                                  "value_frac": tops / (ceiling * world)}
 
     if rank == 0:
         # ---- per-kernel timing (same kernels, same launch configuration, timed one by one)

@@ -480,6 +480,8 @@ def test_benchmark_configs_full_size(spec):
     assert np.array_equal(qw.cpu().numpy(), qw_ref) and np.array_equal(s_ch.cpu().numpy(), s_ch_ref)
     A, bias = t["A"].to(DEV), t["bias"].to(DEV)
     ws = w8.alloc_workspace(M, N, K, w8.ACT_BF16, DEV)
+    if spec.name in ("paper_ffn_down", "paper_llm_proj"):       # deep K and a nearly empty last wave: cut along K
+        assert w8.int8_linear_plan(M, N, K, w8.ACT_BF16, ws.numel())["split_parts"] >= 2
     out = w8.int8_linear_fused(A, qw, s_ch, bias, workspace=ws)
     check_status(ws)
     assert torch.isfinite(out.float()).all()
