@@ -225,7 +225,8 @@ int int8_linear_force_config(int config_id);
  * Reports how int8_linear_fused would run this problem on the current device with a workspace of
  * workspace_bytes (under the forced configuration, if one is set): the kernel configuration, the number
  * of CTAs or CTA pairs launched, and the K-split of the last wave (split_tiles tiles cut into split_parts
- * parts each; both 0 when nothing is cut). Any output pointer may be NULL. Launches nothing.
+ * parts each; both 0 when nothing is cut). Any output pointer may be NULL. Launches nothing and needs no
+ * device (the SM count of the current device is used, 148 if none can be queried).
  */
 int int8_linear_plan(int64_t M, int64_t N, int64_t K, int a_dtype, size_t workspace_bytes,
                      int* config_id, int* cta_groups, int* split_tiles, int* split_parts);

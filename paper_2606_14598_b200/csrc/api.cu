@@ -137,7 +137,7 @@ int int8_linear_plan(int64_t M, int64_t N, int64_t K, int a_dtype, size_t worksp
     const size_t base = int8_linear_workspace_min_bytes(M, N, K, a_dtype);
     if (base == 0) return W8A8_ERR_INVALID_ARG;
     if (workspace_bytes < base) return W8A8_ERR_WORKSPACE;
-    if (int e = check_arch()) return e;          // the plan depends on the device's SM count
+    // no device needed: the plan depends on the SM count only (148 is assumed when no device can be queried)
     const int forced = g_forced_config.load();
     TcPlan plan{};
     if ((forced < 0 && M <= kSkinnyM) || (forced >= 0 && (forced & 0xff) == tc_num_configs())) {

@@ -58,6 +58,36 @@ def test_workspace_sizes():
             assert (hi > lo) == (K == 53248), (M, N, K, lo, hi)
 
 
+def test_plan_of_the_benchmark_shapes():
+    # the static per-shape choice (148 SMs assumed without a device): CTA pairs with 256x256 tiles on the large
+    # shapes; deep K with a nearly empty last wave is cut along K when the workspace has room, and only then
+    w8.force_config(-1)
+    pair = next(i for i in range(w8.num_configs()) if "256x256 per CTA pair" in w8.config_name(i))
+    for (M, N, K) in [(4608, 12288, 3072), (4608, 3072, 12288), (9216, 9216, 3072), (2816, 3072, 3072)]:
+        p = w8.int8_linear_plan(M, N, K, w8.ACT_BF16)
+        assert p["config"] == pair and p["split_parts"] == 0 and p["groups"] == 74, p
+    p = w8.int8_linear_plan(4110, 4608, 53248, w8.ACT_BF16)
+    assert p["config"] == pair and p["groups"] == 74 and p["split_tiles"] == 306 % 74 and p["split_parts"] == 7, p
+    lo = w8.int8_linear_workspace_min_bytes(4110, 4608, 53248, w8.ACT_BF16)
+    assert w8.int8_linear_plan(4110, 4608, 53248, w8.ACT_BF16, lo)["split_parts"] == 0
+    p = w8.int8_linear_plan(512, 4608, 53248, w8.ACT_INT8)
+    assert p["split_parts"] == 2 and p["groups"] == p["split_tiles"] * 2 <= 74, p
+    assert w8.int8_linear_plan(4110, 4608, 4608, w8.ACT_BF16)["split_parts"] == 0       # shallow K: a cut would not pay
+    assert w8.int8_linear_plan(2, 18432, 3072, w8.ACT_BF16)["config"] == w8.num_configs() - 1   # CUDA-core path
+    assert "128x128" in w8.int8_linear_plan(128, 256, 256, w8.ACT_BF16)["name"] or \
+           "256x128" in w8.int8_linear_plan(128, 256, 256, w8.ACT_BF16)["name"]
+    # forcing a configuration cuts whenever it can; + 0x100 never cuts; -2 chooses freely but never cuts
+    w8.force_config(pair)
+    assert w8.int8_linear_plan(256, 512, 2048, w8.ACT_INT8, 64 << 20)["split_parts"] == 2
+    w8.force_config(pair + 0x100)
+    assert w8.int8_linear_plan(256, 512, 2048, w8.ACT_INT8, 64 << 20)["split_parts"] == 0
+    w8.force_config(-2)
+    assert w8.int8_linear_plan(4110, 4608, 53248, w8.ACT_BF16)["split_parts"] == 0
+    w8.force_config(-1)
+    with pytest.raises(w8.W8A8Error):
+        w8.int8_linear_plan(4110, 4608, 53248, w8.ACT_BF16, 1024)                       # below the minimum
+
+
 def test_configs_are_listed():
     n = w8.num_configs()
     assert n >= 2 and all(w8.config_name(i) for i in range(n)) and w8.config_name(n) is None
