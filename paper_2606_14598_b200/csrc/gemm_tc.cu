@@ -8,7 +8,7 @@
 // each CTA loads its own 128 rows of A and its own half (BN/2 rows) of the W tile, the leader CTA
 // issues one MMA for both, and each CTA ends up with its 128 x BN half of the accumulator in its own
 // TMEM. A pair moves half as many W bytes per SM through shared memory as two independent CTAs, which
-// is what the shared-memory bandwidth needs at the int8 rate. No multicast is used anywhere: the
+// is what the shared-memory bandwidth needs at the int8 rate. Every load is a plain per-CTA TMA load: the
 // leader signals the peer's barriers with a second, plain tcgen05.commit / mbarrier.arrive.
 // Warp roles:
 //   warp 0    TMA producer: loads the 128 x 128-byte A tile and the BN x 128-byte
