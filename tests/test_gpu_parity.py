@@ -348,6 +348,44 @@ def test_run_to_run_identical_and_host_buffer_entry_point():
     assert torch.equal(out_host, first.cpu())
 
 
+# ------------------------------------------------------------------------------- stored digests
+
+def test_cuda_results_match_stored_oracle_digests():
+    # tests/golden/oracle_hashes.json holds SHA-256 digests of what the CPU oracle computed from the seeded inputs
+    # (written by tests/golden/make_oracle_hashes.py, which never touches the CUDA library): the device must
+    # produce the same bytes, whatever machine the digests were written on
+    import hashlib
+    import importlib.util
+    import json
+    import os
+    here = os.path.dirname(os.path.abspath(__file__))
+    mspec = importlib.util.spec_from_file_location("make_oracle_hashes", os.path.join(here, "golden", "make_oracle_hashes.py"))
+    mod = importlib.util.module_from_spec(mspec)
+    mspec.loader.exec_module(mod)
+    stored = json.load(open(os.path.join(here, "golden", "oracle_hashes.json")))
+
+    def digest(t):
+        return hashlib.sha256(np.ascontiguousarray(t.cpu().numpy()).tobytes()).hexdigest()
+
+    for spec in mod.CASES:
+        want = stored[spec.name]
+        t = synth.make_linear(spec)
+        assert mod.digest(synth.bf16_bits(t["A"])) == want["A"], "the generator's stream differs on this machine"
+        qw, s_ch = w8.int8_quantize_weight_per_channel(t["W"].to(DEV))
+        bias = None if t["bias"] is None else t["bias"].to(DEV)
+        ws = w8.alloc_workspace(spec.M, spec.N, spec.K, w8.ACT_BF16, DEV)
+        out = w8.int8_linear_fused(t["A"].to(DEV), qw, s_ch, bias, workspace=ws)
+        check_status(ws)
+        s_off, q_off = w8.int8_linear_workspace_offsets(spec.M, spec.K)
+        s_tok = ws[s_off:s_off + 4 * spec.M].view(torch.float32)
+        qa = ws[q_off:q_off + spec.M * spec.K].view(torch.int8).view(spec.M, spec.K)
+        acc = w8.int8_gemm_i32_debug(qa, qw)
+        got = {"qw": digest(qw), "s_ch": digest(s_ch), "qa": digest(qa), "s_tok": digest(s_tok), "acc": digest(acc),
+               "out": digest(out.view(torch.int16))}
+        for key, val in got.items():
+            assert val == want[key], f"{spec.name}: {key}"
+
+
 # ------------------------------------------------------------------------------- K-split of the partial wave
 
 # (M, N, K, configuration): shapes whose last (or only) wave of tiles leaves SMs idle, so that its tiles

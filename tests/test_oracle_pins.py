@@ -361,6 +361,24 @@ def test_generator_is_seeded_and_shaped():
     assert g.float().min() > -0.18 and g.float().max() > 2.0
 
 
+def test_stored_digests_of_inputs_and_oracle_outputs():
+    # tests/golden/oracle_hashes.json was written by tests/golden/make_oracle_hashes.py (generator + oracle only):
+    # the generator's streams and every tensor the oracle derives from them are still bit for bit the same
+    import importlib.util
+    import json
+    import os
+    here = os.path.dirname(os.path.abspath(__file__))
+    spec = importlib.util.spec_from_file_location("make_oracle_hashes", os.path.join(here, "golden", "make_oracle_hashes.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    stored = json.load(open(os.path.join(here, "golden", "oracle_hashes.json")))
+    now = mod.compute_all()
+    assert sorted(now) == sorted(stored)
+    for name in stored:
+        for key in stored[name]:
+            assert now[name][key] == stored[name][key], f"{name}: {key} changed"
+
+
 # --------------------------------------------------------------------------- SmoothQuant hook
 
 def test_smooth_ones_is_plain_and_powers_of_two_are_exact():
