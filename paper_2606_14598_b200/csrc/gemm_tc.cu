@@ -403,7 +403,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             asm volatile("bar.sync 1, 128;" ::: "memory");
             if (ep_tid == 0) *last_flag = atomicAdd(split_counters + unit_slot * CG + rank, 1) == split_s - 1 ? 1 : 0;
             asm volatile("bar.sync 1, 128;" ::: "memory");
-            if (*last_flag == 0 || !ok) return;
+            if (*last_flag == 0) return;               // uniform over the epilogue warps: the barriers below stay matched
             __threadfence();
             // This is the CTA's last piece of work and its MMAs have completed: the operand ring is free. Pull the
             // whole slab into it with asynchronous copies (all in flight at once), then run the usual epilogue.
@@ -411,6 +411,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             for (int i = ep_tid; i < SLAB / 4; i += EPI_THREADS) cp_async_16(base + i * 16, slab + i * 4);
             cp_async_wait_all();
             asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (!ok) return;                           // a wait of this warp gave up: no output from it
             const int32_t* sm_slab = reinterpret_cast<const int32_t*>(base_ptr) + lg * 32 + lane;
 #pragma unroll 1
             for (int cc = 0; cc < CHUNKS; ++cc) {
