@@ -46,7 +46,7 @@ def test_workspace_sizes():
     assert w8.int8_linear_workspace_bytes(8, 8, 16, 5) == 0
     # the smallest accepted workspace is the layout above; the recommended one adds room for the partial sums of
     # the K-split where the shape's last wave of tiles is mostly empty and K is deep (the paper's llm-proj), and
-    # nothing where it is not (the c4 shapes) or where the CUDA-core path runs (M <= 16)
+    # nothing where it is not (the c4 shapes) or where the CUDA-core path runs (M <= 8)
     for (M, N, K) in [(4608, 3072, 12288), (4608, 12288, 3072), (4110, 4608, 53248), (512, 4608, 53248), (2, 18432, 3072)]:
         for dt in (w8.ACT_BF16, w8.ACT_INT8):
             lo, hi = w8.int8_linear_workspace_min_bytes(M, N, K, dt), w8.int8_linear_workspace_bytes(M, N, K, dt)
