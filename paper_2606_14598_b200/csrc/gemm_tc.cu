@@ -20,6 +20,9 @@
 //             scalar per thread; s_ch and bias are per-column broadcasts from
 //             shared memory), dequantize, pack to bf16, stage in swizzled shared
 //             memory, TMA-store 32 x 64 boxes (TMA clips ragged M and N)
+//   warps 6-9 helpers: idle until the CTA's last tile, whose epilogue no k-loop hides;
+//             there they take half of the boxes (a warp reads only the TMEM lanes of
+//             its index modulo 4, so they pair up with warps 2-5 lane group by lane group)
 // Two accumulators of BN columns alternate in TMEM so that the epilogue of one
 // tile overlaps the k-loop of the next. (Eight epilogue warps, two per TMEM lane
 // group, with the per-column scales read straight from global memory, were
@@ -49,8 +52,9 @@ namespace {
 constexpr int BM = 128;            // rows of A per tile (= TMEM lanes)
 constexpr int BK = 128;            // int8 elements (= bytes) of K per stage: one 128-byte swizzle row
 constexpr int MMA_K = 32;          // K of one tcgen05.mma.kind::i8
-constexpr int NUM_THREADS = 192;
-constexpr int EPI_THREADS = 128;
+constexpr int EPI_THREADS = 128;    // warps 2..5: the epilogue of every tile
+constexpr int HELPER_WARP0 = 6;     // warps 6..9: take half of the columns of a CTA's last tile, whose epilogue nothing hides
+constexpr int NUM_THREADS = 64 + 2 * EPI_THREADS;
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;   // 2 s
 
 enum Where { W_PRODUCER_EMPTY = 1, W_MMA_FULL = 2, W_MMA_TMEM_EMPTY = 3, W_EPI_TMEM_FULL = 4 };
@@ -264,23 +268,34 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             if (has_unit && ok) mma_tile(unit_sb, unit_se);
         }
     } else {
-        // ------------------------------------------------------------ epilogue (warps 2..5)
+        // ------------------------------------------------------------ epilogue (warps 2..5, helpers 6..9)
         const int lg = warp & 3;                       // TMEM lane group this warp may read: 32*lg .. 32*lg+31
         const int ep_tid = threadIdx.x - 64;
+        const bool helper = warp >= HELPER_WARP0;
         float* sm_sch = reinterpret_cast<float*>(base_ptr + L::OFF_SCH);
         float* sm_bias = reinterpret_cast<float*>(base_ptr + L::OFF_BIAS);
-        const uint32_t staging = base + L::OFF_STAGING + (warp - 2) * L::STAGING_BYTES_PER_WARP;
-        uint8_t* staging_ptr = base_ptr + L::OFF_STAGING + (warp - 2) * L::STAGING_BYTES_PER_WARP;
+        // staging boxes: the epilogue warps have their own; the helpers borrow the operand ring, which is idle by
+        // the time the last tile's accumulator is complete
+        const int stg_off = helper ? (warp - HELPER_WARP0) * L::STAGING_BYTES_PER_WARP
+                                   : L::OFF_STAGING + (warp - 2) * L::STAGING_BYTES_PER_WARP;
+        const uint32_t staging = base + stg_off;
+        uint8_t* staging_ptr = base_ptr + stg_off;
+        // The epilogue of a CTA's last tile overlaps with nothing: there the helpers take the upper half of the boxes.
+        const int n_regular = tiles_whole > first_tile ? (tiles_whole - first_tile + tile_step - 1) / tile_step : 0;
+        const bool helpers_on = !RAW_I32 && n_regular > 0 && !has_unit;
+        constexpr int ALL_CHUNKS = BN / 32;
+        constexpr int C_SPLIT = 2 * (BN / 64 - BN / 128);            // 32-column chunks the epilogue warps keep on that tile
         const bool has_bias = bias != nullptr;
         const uint64_t stream_out = l2_policy_evict_first();        // the output is written once and not read here
         if (after_quantizer) grid_dep_wait();          // s_tok comes from the kernel before this one
         bool ok = true;
         int it = 0;
         volatile int* last_flag = reinterpret_cast<volatile int*>(base_ptr + L::OFF_LAST);
-        auto epi_tile = [&](int t, bool unit) {
+        // chunks [c_lo, c_hi) of tile t; `shared_tile`: the helpers work on this tile too
+        auto epi_tile = [&](int t, bool unit, int c_lo, int c_hi, bool shared_tile) {
             const int buf = it & 1;
             const int m0 = tile_m(t) * TILE_M + rank * BM, n0 = tile_n(t) * BN;
-            if (!RAW_I32) {
+            if (!RAW_I32 && !helper) {
                 asm volatile("bar.sync 1, 128;" ::: "memory");     // previous tile's readers are done
                 for (int j = ep_tid; j < BN; j += EPI_THREADS) {
                     const int n = n0 + j;
@@ -289,6 +304,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 }
                 asm volatile("bar.sync 1, 128;" ::: "memory");
             }
+            // the helpers have been parked here since the start of the kernel: the scales of the last tile are in place
+            if (shared_tile) asm volatile("bar.sync 2, 256;" ::: "memory");
             const int row = m0 + lg * 32 + lane;
             const float st = (!RAW_I32 && row < M) ? __ldg(s_tok + row) : 0.f;
             if (ok && !mbar_wait(tfull_bar(buf), (it >> 1) & 1, ctl, W_EPI_TMEM_FULL, kStatusTimeout)) ok = false;
@@ -353,22 +370,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             auto release_accumulator = [&]() {         // every TMEM load of this tile has completed
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) {
+                if (lane == 0 && !helper) {            // (nothing follows a tile the helpers work on)
                     if (CG == 2) mbar_arrive_cluster(mapa_shared(tempty_bar(buf), 0));
                     else mbar_arrive(tempty_bar(buf));
                 }
             };
-            constexpr int CHUNKS = BN / 32;
+            constexpr int CHUNKS = ALL_CHUNKS;
             uint32_t va[32], vb[32];
             if (!unit) {
-                tmem_ld_32x32b_x32(t_row, va);
+                tmem_ld_32x32b_x32(t_row + c_lo * 32, va);
 #pragma unroll 1
-                for (int cc = 0; cc < CHUNKS; cc += 2) {
+                for (int cc = c_lo; cc < c_hi; cc += 2) {
                     tmem_wait_ld();
                     tmem_ld_32x32b_x32(t_row + (cc + 1) * 32, vb);
                     process(cc, va);
                     tmem_wait_ld();
-                    if (cc + 2 < CHUNKS) tmem_ld_32x32b_x32(t_row + (cc + 2) * 32, va);
+                    if (cc + 2 < c_hi) tmem_ld_32x32b_x32(t_row + (cc + 2) * 32, va);
                     else release_accumulator();
                     process(cc + 1, vb);
                 }
@@ -420,8 +437,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 process(cc, va);
             }
         };
-        for (int t = first_tile; t < tiles_whole; t += tile_step, ++it) epi_tile(t, false);
-        if (has_unit) epi_tile(unit_tile, true);
+        if (!helper) {
+            for (int t = first_tile; t < tiles_whole; t += tile_step, ++it) {
+                const bool shared_tile = helpers_on && it == n_regular - 1;
+                epi_tile(t, false, 0, shared_tile ? C_SPLIT : ALL_CHUNKS, shared_tile);
+            }
+            if (has_unit) epi_tile(unit_tile, true, 0, ALL_CHUNKS, false);
+        } else if (helpers_on) {
+            it = n_regular - 1;
+            epi_tile(first_tile + it * tile_step, false, C_SPLIT, ALL_CHUNKS, true);
+        }
         if (!RAW_I32 && lane == 0) bulk_wait_group<0>();
     }
 
