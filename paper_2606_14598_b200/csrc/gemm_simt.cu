@@ -27,8 +27,6 @@ gemm_simt_kernel(const int8_t* __restrict__ qa, int64_t lda_q, const float* __re
                  const int8_t* __restrict__ qw, const float* __restrict__ s_ch, const float* __restrict__ bias,
                  void* __restrict__ out, int64_t ldo, int M, int N, int K, int raw_i32, int after_quantizer, int* status) {
     grid_dep_launch_dependents();      // a following kernel launched to allow it may set itself up early
-    // no quantizer ahead of this kernel to clear the status word: do it here (this kernel has no waits that could set it)
-    if (!after_quantizer && status != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *status = 0;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n0 = (blockIdx.x * WARPS + warp) * NPW;
     const int m0 = blockIdx.y * MB;
@@ -47,8 +45,10 @@ gemm_simt_kernel(const int8_t* __restrict__ qa, int64_t lda_q, const float* __re
 #pragma unroll
     for (int i = 0; i < MB; ++i) arow[i] = qa + static_cast<int64_t>(min(m0 + i, M - 1)) * lda_q;
 
-    // weights do not depend on the quantizer: warm the first chunk before waiting for it
-    if (after_quantizer) grid_dep_wait();
+    // always launched so that it may start while the kernel ahead of it is finishing: wait for that kernel's results
+    grid_dep_wait();
+    // no quantizer ahead of this kernel to clear the status word: do it here (this kernel has no waits that could set it)
+    if (!after_quantizer && status != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && warp == 0 && lane == 0) *status = 0;
 
 #pragma unroll 2
     for (int k = lane * 16; k < K; k += 32 * 16) {      // unrolled: several 512-byte slices of each weight row in flight
@@ -104,7 +104,7 @@ cudaError_t launch(const GemmArgs& a, cudaStream_t st) {
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = a.after_quantizer ? 1 : 0;
+    cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, gemm_simt_kernel<MB, NPW, WARPS>, a.qa, a.lda_q, a.s_tok, a.qw, a.s_ch, a.bias,
                               a.out, a.ldo, a.M, a.N, a.K, a.raw_i32 ? 1 : 0, a.after_quantizer ? 1 : 0, a.status);
 }

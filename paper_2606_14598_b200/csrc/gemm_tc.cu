@@ -123,9 +123,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     constexpr uint32_t TMEM_COLS = 2 * TMEM_BUF;
     static_assert(BN % 64 == 0 && BN <= 256, "BN: whole 64-column output boxes, at most 256 TMEM columns per buffer");
 
-    // without a quantizer ahead of it (which clears the status word) the kernel clears it itself; a time-out
-    // can only be recorded seconds later
-    if (!after_quantizer && blockIdx.x == 0 && threadIdx.x == 0) *status = 0;
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             for (int sub = 0; sub < KBS; ++sub) mbar_init(full_bar(s, sub), 1);
@@ -168,7 +165,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     auto tile_m = [&](int t) { return t / num_n; };
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer (both CTAs of a pair)
-        if (after_quantizer && lane == 0) grid_dep_wait();   // qa comes from the kernel before this one
+        // The kernel is always launched so that it may start while the kernel ahead of it in the stream is finishing
+        // (the quantizer, or whatever the caller ran): everything up to here touched no global memory.
+        if (lane == 0) {
+            grid_dep_wait();
+            // without a quantizer ahead of it (which clears the status word) the kernel clears it itself; a time-out
+            // can only be recorded seconds later
+            if (!after_quantizer && blockIdx.x == 0) *status = 0;
+        }
         __syncwarp();
         int stage = 0;
         uint32_t phase = 0;
@@ -287,7 +291,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         constexpr int C_SPLIT = 2 * (BN / 64 - BN / 128);            // 32-column chunks the epilogue warps keep on that tile
         const bool has_bias = bias != nullptr;
         const uint64_t stream_out = l2_policy_evict_first();        // the output is written once and not read here
-        if (after_quantizer) grid_dep_wait();          // s_tok comes from the kernel before this one
+        grid_dep_wait();                               // s_tok may come from the kernel before this one
         bool ok = true;
         int it = 0;
         volatile int* last_flag = reinterpret_cast<volatile int*>(base_ptr + L::OFF_LAST);
@@ -553,11 +557,9 @@ int launch_cfg(const GemmArgs& a, const TcPlan& plan, cudaStream_t st) {
         attr[na].val.clusterDim.z = 1;
         ++na;
     }
-    if (a.after_quantizer) {
-        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[na].val.programmaticStreamSerializationAllowed = 1;
-        ++na;
-    }
+    attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
     cfg.attrs = attr;
     cfg.numAttrs = na;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tm_a, tm_b, tm_out, a.s_tok, a.s_ch, a.bias,
