@@ -27,8 +27,8 @@ if ROOT not in sys.path:
 
 METRIC = "fused W8A8 linear TOPS (% of B200 dense INT8 peak) per DiT GEMM shape"
 INT8_PEAK_TOPS = 4500.0            # B200 datasheet, dense INT8
-# measured DRAM traffic of one gemm_tc_kernel launch (ncu, see profiles/): c4 = mean of up (138.9 MB) and down (135.1 MB)
-NCU_GEMM_DRAM_BYTES_PER_LAUNCH = {"c4": 137.0e6}
+# measured DRAM traffic of one gemm_tc_kernel launch (ncu, see profiles/): c4 = mean of up (138.8 MB) and down (136.9 MB)
+NCU_GEMM_DRAM_BYTES_PER_LAUNCH = {"c4": 137.85e6}
 L2_BYTES = 126 * 1024 * 1024
 
 
