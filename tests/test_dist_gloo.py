@@ -69,3 +69,25 @@ def test_shard_rows_partition():
                 assert all(a[1] == b[0] for a, b in zip(spans, spans[1:]))
                 sizes = [hi - lo for lo, hi in spans]
                 assert max(sizes) - min(sizes) <= 2 * mult - 1
+
+
+def test_reference_arm_prints_one_json_line_and_only_on_rank_zero():
+    # `bench.py --impl reference` times the CPU oracle and needs no GPU; launched as ranks of a multi-process job,
+    # rank 0 alone does the work and prints, the others leave at once
+    import json
+    cmd = [sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "c1", "--steps", "1", "--warmup", "0"]
+    env = dict(os.environ, OMP_NUM_THREADS="2")
+    for k in ("RANK", "LOCAL_RANK", "WORLD_SIZE"):
+        env.pop(k, None)
+    r = subprocess.run(cmd, env=env, capture_output=True, text=True, timeout=300, cwd=ROOT)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.strip()]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["impl"] == "reference" and d["unit"] == "TOPS" and d["value"] > 0 and d["higher_is_better"] is True
+    assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] >= 1 and d["cpu_baseline"]["sample"]
+    assert d["e2e"]["h2d_bytes_per_step"] == 0 and d["e2e"]["d2h_bytes_per_step"] == 0 and d["gpu_launches"] == 0
+    assert d["config"]["workload"].startswith("c1")
+    env1 = dict(env, RANK="1", LOCAL_RANK="1", WORLD_SIZE="2", MASTER_ADDR="127.0.0.1", MASTER_PORT=str(free_port()))
+    r1 = subprocess.run(cmd + ["--gpus", "2"], env=env1, capture_output=True, text=True, timeout=300, cwd=ROOT)
+    assert r1.returncode == 0 and r1.stdout.strip() == "", r1.stderr[-2000:]
