@@ -453,6 +453,42 @@ def test_k_split_from_bf16_automatic_choice():
     assert torch.equal(out, out2)
 
 
+# ------------------------------------------------------------------------------- random shapes, every configuration
+
+def test_random_shapes_all_configurations_agree_with_the_cuda_core_path():
+    # 40 seeded random shapes (ragged in every dimension, K tails inside a pipeline stage, one to a few hundred
+    # tiles). The CUDA-core path is checked against the oracle on the first 12; every tensor-core configuration,
+    # with and without the K-split, must then give the same accumulators and the same output bits as that path.
+    rng = np.random.default_rng(2606)
+    simt = n_tc_configs()
+    big_ws = torch.empty(48 << 20, dtype=torch.uint8, device=DEV)
+    for case in range(40):
+        M = int(rng.integers(1, 700))
+        N = 8 * int(rng.integers(1, 190))
+        K = 16 * int(rng.integers(1, 380))
+        qa, qw = rand_codes(rng, (M, K)), rand_codes(rng, (N, K))
+        s_tok = (rng.random(M) * 0.05 + 0.01).astype(np.float32)
+        s_ch = (rng.random(N) * 0.0008 + 0.0002).astype(np.float32)
+        bias = (rng.standard_normal(N) * 0.01).astype(np.float32)
+        dev = [torch.from_numpy(a).to(DEV) for a in (qa, qw, s_tok, s_ch, bias)]
+        w8.force_config(simt)
+        acc_ref = w8.int8_gemm_i32_debug(dev[0], dev[1], big_ws)
+        out_ref = w8.int8_linear_fused(dev[0], dev[1], dev[3], dev[4], s_tok=dev[2], workspace=big_ws).clone()
+        check_status(big_ws)
+        if case < 12:
+            ref = oracle.linear_fused_int8(qa, s_tok, qw, s_ch, bias)
+            assert np.array_equal(acc_ref.cpu().numpy(), ref["acc"]), (M, N, K)
+            assert_bf16_close(synth.bf16_bits(out_ref.cpu()), ref["out"])
+        for cfg in range(simt):
+            for forced in (cfg, cfg + 0x100):
+                w8.force_config(forced)
+                acc = w8.int8_gemm_i32_debug(dev[0], dev[1], big_ws)
+                out = w8.int8_linear_fused(dev[0], dev[1], dev[3], dev[4], s_tok=dev[2], workspace=big_ws)
+                check_status(big_ws)
+                assert torch.equal(acc, acc_ref), (M, N, K, forced)
+                assert torch.equal(out, out_ref), (M, N, K, forced)
+
+
 # ------------------------------------------------------------------------------- CUDA graph of a block's linears
 
 def test_cuda_graph_replay_of_several_linears():
