@@ -489,6 +489,32 @@ def test_random_shapes_all_configurations_agree_with_the_cuda_core_path():
                 assert torch.equal(out, out_ref), (M, N, K, forced)
 
 
+# ------------------------------------------------------------------------------- two streams
+
+def test_two_streams_with_their_own_workspaces_do_not_disturb_each_other():
+    # calls on different streams may overlap on the device as long as each has its own workspace
+    specs = [synth.LinearSpec("s0", 700, 1024, 1544), synth.LinearSpec("s1", 520, 8192, 776)]   # the second one is cut along K
+    lanes = []
+    for spec in specs:
+        t = synth.make_linear(spec)
+        qw, s_ch = w8.int8_quantize_weight_per_channel(t["W"].to(DEV))
+        A, bias = t["A"].to(DEV), t["bias"].to(DEV)
+        ws = w8.alloc_workspace(spec.M, spec.N, spec.K, w8.ACT_BF16, DEV)
+        want = w8.int8_linear_fused(A, qw, s_ch, bias, workspace=ws).clone()
+        check_status(ws)
+        lanes.append({"A": A, "qw": qw, "s_ch": s_ch, "bias": bias, "ws": ws, "want": want,
+                      "out": torch.empty_like(want), "stream": torch.cuda.Stream(DEV)})
+    torch.cuda.synchronize()
+    for _ in range(25):
+        for L in lanes:
+            with torch.cuda.stream(L["stream"]):
+                w8.int8_linear_fused(L["A"], L["qw"], L["s_ch"], L["bias"], out=L["out"], workspace=L["ws"])
+    torch.cuda.synchronize()
+    for L in lanes:
+        check_status(L["ws"])
+        assert torch.equal(L["out"], L["want"])
+
+
 # ------------------------------------------------------------------------------- CUDA graph of a block's linears
 
 def test_cuda_graph_replay_of_several_linears():
