@@ -499,9 +499,22 @@ def main():
                 s_off, q_off = w8.int8_linear_workspace_offsets(spec.M, spec.K)
                 qa = L["ws"][q_off:q_off + spec.M * spec.K].view(torch.int8).view(spec.M, spec.K)
                 ti = statistics.mean(cuda_timer(torch, lambda: torch._int_mm(qa, L["qw"].t()), 10, 3))
+                # the unfused route the paper compares with: library integer matmul, then a separate dequantization pass
+                s_tok_v = L["ws"][s_off:s_off + 4 * spec.M].view(torch.float32)
+
+                def unfused():
+                    acc = torch._int_mm(qa, L["qw"].t())
+                    y = acc.float() * s_tok_v[:, None] * L["s_ch"][None, :]
+                    if L["bias"] is not None:
+                        y = y + L["bias"][None, :]
+                    return y.to(torch.bfloat16)
+
+                tu = statistics.mean(cuda_timer(torch, unfused, 6, 2))
                 mine = next(p for p in per_shape if p["name"] == spec.name)
                 ctx.append({"name": spec.name, "torch_bf16_matmul_tflops": spec.ops / tb / 1e12,
                             "torch_int_mm_tops_no_dequant": spec.ops / ti / 1e12,
+                            "unfused_int_mm_plus_dequant_us": tu * 1e6,
+                            "gemm_epilogue_speedup_over_unfused": tu / (mine["gemm_epilogue_us"] * 1e-6),
                             # the paper's Table 1 quantity on this machine: fused int8 linear over library bf16 matmul
                             "fused_from_bf16_speedup_over_bf16_matmul": tb / (mine["fused_from_bf16_us"] * 1e-6),
                             "gemm_epilogue_speedup_over_bf16_matmul": tb / (mine["gemm_epilogue_us"] * 1e-6)})
