@@ -153,7 +153,7 @@ def run_reference(args):
     if rank != 0:
         return
     from paper_2606_14598_b200 import inputs as synth
-    specs = synth.CONFIGS[args.workload]
+    specs = workload_specs(args)
     steps, warmup = max(1, min(args.steps, 3)), min(args.warmup, 1)
     tops, sec, cores, sample = time_oracle(specs, steps, warmup, target_gmac=20.0)
     line = {
@@ -174,6 +174,17 @@ def workload_name(key, specs):
 
 
 # ------------------------------------------------------------------------------------------ CUDA arm
+
+def workload_specs(args):
+    """The linears of the chosen workload, with the token count overridden if asked (skinny linears keep theirs)."""
+    import dataclasses
+
+    from paper_2606_14598_b200 import inputs as synth
+    specs = synth.CONFIGS[args.workload]
+    if args.rows > 0:
+        specs = [s if s.M <= 16 else dataclasses.replace(s, M=args.rows, name=f"{s.name}_m{args.rows}") for s in specs]
+    return specs
+
 
 def cuda_timer(torch, fn, iters, warm):
     for _ in range(warm):
@@ -197,6 +208,8 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--sets", type=int, default=3, help="rotating input/weight sets (keeps steps out of L2)")
     ap.add_argument("--no-extras", action="store_true", help="skip e2e, context and CPU-baseline legs")
+    ap.add_argument("--rows", type=int, default=0,
+                    help="override the token count M of every linear of the workload (the paper sweeps M = 512 ... 16384)")
     ap.add_argument("--launch", default="direct", choices=["graph", "direct"],
                     help="graph: each step is one replay of a captured CUDA graph of the step's calls; direct: the calls themselves")
     ap.add_argument("--config", type=int, default=-1, help="force a kernel configuration (sweeps); -1 = from the shape")
@@ -217,7 +230,7 @@ def main():
     rank, local_rank, world = wdist.init("nccl")
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    specs = synth.CONFIGS[args.workload]
+    specs = workload_specs(args)
     peaks = measured_peaks()
     w8.force_config(args.config)
 
