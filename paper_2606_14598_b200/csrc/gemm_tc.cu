@@ -515,25 +515,14 @@ constexpr size_t kCounterBytes = 1024;    // per-tile arrival counters at the he
 constexpr int kMaxSplit = 8;              // parts per tile
 constexpr int kMinStagesPerPart = 4;
 
-int sm_count() {
-    static int n = [] {
-        int dev = 0, v = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
-        return v > 0 ? v : 148;
-    }();
-    return n;
-}
-
 template <int CG, int BN, int STAGES, int KBS, bool RAW>
 int launch_cfg(const GemmArgs& a, const TcPlan& plan, cudaStream_t st) {
     using L = SmemLayout<CG, BN, STAGES, KBS>;
     static_assert(L::DYN_BYTES <= 232448, "shared memory budget");
     auto kern = gemm_tc_kernel<CG, BN, STAGES, KBS, RAW>;
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(once, [&] { attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES); });
-    if (attr_err != cudaSuccess) return 6;
+    static PerDeviceOnce smem_opt_in;
+    if (smem_opt_in.run([&] { return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES); }) != cudaSuccess)
+        return 6;
 
     CUtensorMap tm_a, tm_b, tm_out;
     if (!encode_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, a.qa, a.M, a.K, a.lda_q, BM, BK)) return 6;

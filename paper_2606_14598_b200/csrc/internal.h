@@ -5,7 +5,47 @@
 #include <cstdint>
 #include <cuda_runtime.h>
 
+#include <mutex>
+
 namespace w8a8 {
+
+// Function attributes (the opt-in to large dynamic shared memory) belong to a device: `set` runs once for every
+// device a launch is made on, under a lock, and its result is remembered.
+class PerDeviceOnce {
+public:
+    template <typename F>
+    cudaError_t run(F&& set) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+        std::lock_guard<std::mutex> lock(mutex_);
+        if (!done_[dev]) {
+            err_[dev] = set();
+            done_[dev] = true;
+        }
+        return err_[dev];
+    }
+
+private:
+    static constexpr int kMaxDevices = 64;
+    std::mutex mutex_;
+    bool done_[kMaxDevices] = {};
+    cudaError_t err_[kMaxDevices] = {};
+};
+
+// SM count of the current device (148 if no device can be queried, so that host-only planning still works).
+inline int sm_count() {
+    static std::mutex mutex;
+    static int cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    std::lock_guard<std::mutex> lock(mutex);
+    if (cached[dev] == 0) {
+        int v = 0;
+        cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
+        cached[dev] = v > 0 ? v : 148;
+    }
+    return cached[dev];
+}
 
 // Device-side status codes written into the workspace status word (low byte
 // is a w8a8_status value, the next byte says which wait gave up).

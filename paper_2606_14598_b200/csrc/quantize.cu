@@ -444,16 +444,6 @@ cudaError_t launch_pdl(void (*kern)(KArgs...), int grid, int block, size_t smem,
     return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
 }
 
-int sm_count() {
-    static int n = [] {
-        int dev = 0, v = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
-        return v > 0 ? v : 148;
-    }();
-    return n;
-}
-
 template <typename T, int WPR>
 cudaError_t launch_reg(const T* x, int64_t ld, int rows, int K, int8_t* q, float* s, int* status, const float* mult,
                        cudaStream_t st) {
@@ -494,14 +484,14 @@ cudaError_t launch_staged(const __nv_bfloat16* x, int64_t ld, int rows, int K, i
     // the ring indices of the kernel wrap at num_stages: a ring of fewer than two stages must never be launched
     if (num_stages < 2) return cudaErrorInvalidConfiguration;
     const int smem = num_stages * stage_bytes + 16 * num_stages + SG_WARPS * 4 + 16 + 128;
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(once, [] {
-        attr_err = cudaFuncSetAttribute(quant_rows_staged_kernel<WPR, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        SG_SMEM_MAX);
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(quant_rows_staged_kernel<WPR, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            SG_SMEM_MAX);
+    static PerDeviceOnce smem_opt_in;
+    const cudaError_t attr_err = smem_opt_in.run([] {
+        cudaError_t e = cudaFuncSetAttribute(quant_rows_staged_kernel<WPR, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             SG_SMEM_MAX);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(quant_rows_staged_kernel<WPR, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     SG_SMEM_MAX);
+        return e;
     });
     if (attr_err != cudaSuccess) return attr_err;
     const int cap = ctas_per_sm * sm_count();
