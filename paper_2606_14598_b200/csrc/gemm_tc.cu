@@ -38,6 +38,7 @@
 // Every mbarrier wait is bounded: on expiry the CTA records W8A8_ERR_TIMEOUT in
 // the workspace status word, all roles unwind, TMEM is freed and the kernel
 // returns.
+#include "../../include/w8a8_linear.h"
 #include "internal.h"
 #include "ptx.cuh"
 
@@ -522,15 +523,15 @@ int launch_cfg(const GemmArgs& a, const TcPlan& plan, cudaStream_t st) {
     auto kern = gemm_tc_kernel<CG, BN, STAGES, KBS, RAW>;
     static PerDeviceOnce smem_opt_in;
     if (smem_opt_in.run([&] { return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES); }) != cudaSuccess)
-        return 6;
+        return W8A8_ERR_CUDA;
 
     CUtensorMap tm_a, tm_b, tm_out;
-    if (!encode_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, a.qa, a.M, a.K, a.lda_q, BM, BK)) return 6;
-    if (!encode_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, a.qw, a.N, a.K, a.K, L::B_ROWS, BK)) return 6;
+    if (!encode_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, a.qa, a.M, a.K, a.lda_q, BM, BK)) return W8A8_ERR_CUDA;
+    if (!encode_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, a.qw, a.N, a.K, a.K, L::B_ROWS, BK)) return W8A8_ERR_CUDA;
     if (RAW) {
         tm_out = tm_a;   // unused
     } else {
-        if (!encode_2d(&tm_out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, a.out, a.M, a.N, a.ldo * 2, 32, 64)) return 6;
+        if (!encode_2d(&tm_out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, a.out, a.M, a.N, a.ldo * 2, 32, 64)) return W8A8_ERR_CUDA;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(CG * plan.groups);
@@ -556,7 +557,7 @@ int launch_cfg(const GemmArgs& a, const TcPlan& plan, cudaStream_t st) {
                                        a.after_quantizer ? 1 : 0, plan.split_tiles, plan.split_parts,
                                        reinterpret_cast<int32_t*>(static_cast<uint8_t*>(a.split_ws) + kCounterBytes),
                                        static_cast<int*>(a.split_ws));
-    return e == cudaSuccess ? 0 : 6;
+    return e == cudaSuccess ? W8A8_OK : W8A8_ERR_CUDA;
 }
 
 template <bool RAW>
@@ -567,7 +568,7 @@ int launch_by_id(const GemmArgs& a, const TcPlan& plan, cudaStream_t st) {
         case 2: return launch_cfg<2, 256, 3, 2, RAW>(a, plan, st);
         case 3: return launch_cfg<2, 128, 4, 2, RAW>(a, plan, st);
         case 4: return launch_cfg<2, 192, 3, 2, RAW>(a, plan, st);
-        default: return 1;
+        default: return W8A8_ERR_INVALID_ARG;
     }
 }
 
@@ -648,7 +649,7 @@ size_t tc_max_scratch_bytes(int M, int N, int K) {
 }
 
 int launch_gemm_tc(const GemmArgs& a, const TcPlan& plan, cudaStream_t st) {
-    if (plan.split_parts >= 2 && a.split_ws == nullptr) return 1;
+    if (plan.split_parts >= 2 && a.split_ws == nullptr) return W8A8_ERR_INVALID_ARG;
     return a.raw_i32 ? launch_by_id<true>(a, plan, st) : launch_by_id<false>(a, plan, st);
 }
 
