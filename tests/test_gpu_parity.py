@@ -317,6 +317,25 @@ def test_fused_from_int8_with_row_stride_and_guard_bands():
         assert (canvas[mask] == SENT).all(), f"config {cfg} wrote outside its output"
 
 
+def test_fused_from_bf16_with_row_stride_no_bias_and_k_split():
+    # activations that are a column slice of a wider tensor (row stride > K), no bias, on a shape that is cut along K
+    spec = synth.LinearSpec("strided", 260, 8192, 520, bias=False)
+    t = synth.make_linear(spec)
+    qw_ref, s_ch_ref = oracle.quantize_weight_per_channel(t["W"].numpy())
+    ref = oracle.linear_fused_bf16(synth.bf16_bits(t["A"]), qw_ref, s_ch_ref, None)
+    qw, s_ch = w8.int8_quantize_weight_per_channel(t["W"].to(DEV))
+    wide = torch.full((spec.M, spec.K + 72), 7.0, dtype=torch.bfloat16, device=DEV)
+    wide[:, 8:8 + spec.K] = t["A"].to(DEV)
+    A_view = wide[:, 8:8 + spec.K]
+    assert A_view.stride(0) == spec.K + 72 and A_view.data_ptr() % 16 == 0
+    ws = w8.alloc_workspace(spec.M, spec.N, spec.K, w8.ACT_BF16, DEV)
+    assert w8.int8_linear_plan(spec.M, spec.N, spec.K, w8.ACT_BF16, ws.numel())["split_parts"] >= 2
+    out = w8.int8_linear_fused(A_view, qw, s_ch, None, workspace=ws)
+    check_status(ws)
+    assert_bf16_close(synth.bf16_bits(out.cpu()), ref["out"])
+    assert (wide[:, :8] == 7.0).all() and (wide[:, 8 + spec.K:] == 7.0).all()
+
+
 @pytest.mark.parametrize("M", [1, 2, 5, 16])
 def test_skinny_m_path(M):
     spec = synth.LinearSpec(f"skinny{M}", M, 3072, 2048, outlier_frac=0.0)
