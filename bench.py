@@ -369,6 +369,8 @@ def main():
         "dtype": "int8", "data": "synthetic",
         "config": {"workload": workload_name(args.workload, specs), "entry": "int8_linear_fused from bf16 activations",
                    "launch": launch_note,
+                   "regime": "one loop of --steps steps; beyond ~200 steps (50 ms) the 1 kW power cap sets the clock "
+                             "(see clocks); the first 100 steps are reported as burst",
                    "l2": f"inputs larger than L2: {len(sets)} rotating sets of {set_bytes / 1e6:.0f} MB each",
                    "parallelism": f"dp{world} over tokens, weights replicated, no collective"},
         "pct_of_int8_peak": 100.0 * tops / (INT8_PEAK_TOPS * world), "int8_peak_tops": INT8_PEAK_TOPS,
