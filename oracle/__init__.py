@@ -78,27 +78,42 @@ def _chk(a, dtype, ndim):
     return a
 
 
+def _chk_rows(a, dtype):
+    """Rank-2 array whose rows are contiguous; the rows themselves may be a fixed number of elements apart
+    (a column slice of a wider C-contiguous array). Returns (array, row stride in elements)."""
+    a = np.asarray(a)
+    if a.dtype != dtype or a.ndim != 2:
+        raise TypeError(f"expected {dtype} array of rank 2, got {a.dtype} {a.shape}")
+    item = a.dtype.itemsize
+    if a.shape[1] > 1 and a.strides[1] != item:
+        raise TypeError("rows must be contiguous")
+    ld = a.strides[0] // item if a.shape[0] > 1 else a.shape[1]
+    if a.shape[0] > 1 and (a.strides[0] % item != 0 or ld < a.shape[1]):
+        raise TypeError("row stride must be a whole number of elements, at least the row length")
+    return a, ld
+
+
 def num_threads() -> int:
     return int(_load().oracle_num_threads())
 
 
 def quantize_weight_per_channel(W: np.ndarray):
-    """fp32 [N,K] -> (int8 [N,K], fp32 [N])."""
-    W = _chk(W, np.float32, 2)
+    """fp32 [N,K] (rows may be strided: a column slice of a wider array) -> (int8 [N,K], fp32 [N])."""
+    W, ldw = _chk_rows(W, np.float32)
     N, K = W.shape
     qw = np.empty((N, K), np.int8)
     s_ch = np.empty((N,), np.float32)
-    _load().oracle_quantize_weight_per_channel(_p(W), N, K, K, _p(qw), _p(s_ch))
+    _load().oracle_quantize_weight_per_channel(_p(W), N, K, ldw, _p(qw), _p(s_ch))
     return qw, s_ch
 
 
 def quantize_act_per_token(A_bits: np.ndarray):
-    """bf16 bit patterns uint16 [M,K] -> (int8 [M,K], fp32 [M])."""
-    A_bits = _chk(A_bits, np.uint16, 2)
+    """bf16 bit patterns uint16 [M,K] (rows may be strided) -> (int8 [M,K], fp32 [M])."""
+    A_bits, lda = _chk_rows(A_bits, np.uint16)
     M, K = A_bits.shape
     qa = np.empty((M, K), np.int8)
     s_tok = np.empty((M,), np.float32)
-    _load().oracle_quantize_act_per_token(_p(A_bits), M, K, K, _p(qa), _p(s_tok))
+    _load().oracle_quantize_act_per_token(_p(A_bits), M, K, lda, _p(qa), _p(s_tok))
     return qa, s_tok
 
 

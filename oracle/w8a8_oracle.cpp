@@ -18,8 +18,11 @@
 //     acc  = sum_k qa[m,k] * qw[n,k]            exact integer
 //     t    = float(acc); t = t * s_tok[m]; t = t * s_ch[n]; t = t + bias[n]
 //     out  = bf16_rne(t)
-// Roundings to integer and to bf16 are done on values / bit patterns directly,
-// never through the floating-point environment.
+// The roundings to integer (codes) and to bf16 (outputs) are done on values / bit
+// patterns directly. The arithmetic itself (/, *, +, and the int32 -> fp32
+// conversion float(acc)) is the compiler's IEEE binary32 in the default
+// round-to-nearest-even mode, with contraction off; the 2^24 and 2^31 edge
+// vectors in the pins check that conversion.
 //
 // Pins (see tests/test_oracle_pins.py): hand tie vectors for the quantizer,
 // scaling / sign / permutation invariants, brute force over tiny shapes,
@@ -28,7 +31,7 @@
 // matmul as outliers vanish. Parity against the authors' own tensors is
 // unpinned: the paper prints no tensor values.
 //
-// Build: g++ -O2 -fopenmp -ffp-contract=off -shared -fPIC (see oracle/build.py)
+// Build: g++ -O2 -fopenmp -ffp-contract=off -fno-fast-math -shared -fPIC (build() in oracle/__init__.py)
 
 #include <cstdint>
 #include <cstring>

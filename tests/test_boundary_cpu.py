@@ -147,3 +147,33 @@ def test_no_device_means_a_loud_error_not_a_fallback():
         pytest.skip("a GPU is present")
     # valid arguments, no device: the call must fail (CUDA error), never compute on the CPU
     assert fused() in (5, 6)
+
+
+def test_oracle_side_processes_do_not_map_the_cuda_library():
+    # The generator, the work model, the multi-rank plumbing and the oracle must run in a process that never
+    # maps libw8a8_linear.so (the oracle's independence is only worth something if its processes are free of
+    # the product); the library is loaded by the first touch of a compute entry point, and only then.
+    import subprocess
+    import sys
+    import textwrap
+    code = textwrap.dedent("""
+        import sys
+        sys.path.insert(0, %r)
+        import numpy as np
+        import oracle
+        import paper_2606_14598_b200 as pkg
+        from paper_2606_14598_b200 import inputs, roofline, dist
+        t = inputs.make_linear(inputs.LinearSpec("indep", 8, 32, 16))
+        qw, s_ch = oracle.quantize_weight_per_channel(t["W"].numpy())
+        out = oracle.linear_fused_bf16(inputs.bf16_bits(t["A"]), qw, s_ch, t["bias"].numpy())["out"]
+        assert out.shape == (8, 16) and roofline.ops(8, 16, 32) == 8192 and dist.shard_rows(8, 0, 2) == (0, 4)
+        maps = open("/proc/self/maps").read()
+        assert "libw8a8_oracle" in maps
+        assert "libw8a8_linear" not in maps, "the CUDA library was mapped by an oracle-side import"
+        assert "paper_2606_14598_b200.binding" not in sys.modules
+        pkg.status_string(0)                         # first touch of an entry point loads it
+        assert "libw8a8_linear" in open("/proc/self/maps").read()
+        print("independent")
+    """) % ROOT
+    r = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0 and "independent" in r.stdout, r.stdout + r.stderr

@@ -128,13 +128,33 @@ def test_quantizer_invariants():
 
 
 def test_quantizer_leading_dimension_is_honoured():
-    # the ctypes wrapper passes dense arrays; check rows do not bleed into each other
+    # rows do not bleed into each other (dense case, hand values)
     x = np.zeros((2, 8), np.float32)
     x[0] = [1, 2, 3, 4, 5, 6, 7, 8]
     x[1] = [-80, 0, 0, 0, 0, 0, 0, 40]
     q, s = oracle.quantize_weight_per_channel(x)
     assert s[0] == f32(8) / f32(127) and s[1] == f32(80) / f32(127)
     assert q[0, 7] == 127 and q[1, 0] == -127 and q[1, 7] in (63, 64)
+    # a row stride larger than the row: the matrix is a column slice of a wider one whose other columns hold
+    # values that would change every scale if they were read (1000 > any |x|), and would shift every code if the
+    # stride were taken for the row length
+    wide = np.full((3, 8 + 5), 1000.0, np.float32)
+    wide[:, 2:10] = [[1, 2, 3, 4, 5, 6, 7, 127], [-127, 0.5, 1.5, 2.5, 0, 0, 0, 0], [0, 0, 0, 0, 0, 0, 0, 0]]
+    view = wide[:, 2:10]
+    assert view.strides == (13 * 4, 4) and not view.flags["C_CONTIGUOUS"]
+    q, s = oracle.quantize_weight_per_channel(view)
+    assert s.tolist() == [1.0, 1.0, 1.0]
+    assert q.tolist() == [[1, 2, 3, 4, 5, 6, 7, 127], [-127, 0, 2, 2, 0, 0, 0, 0], [0] * 8]
+    # the same through the bf16 entry, and against the dense copy on random data
+    rng = np.random.default_rng(17)
+    a = rng.standard_normal((9, 40 + 24)).astype(np.float32)
+    a[:, :3] *= 50                                          # outside the slice: larger than anything inside
+    bits_wide = bf16_bits_of(a)
+    sl = bits_wide[:, 8:48]
+    qd, sd = oracle.quantize_act_per_token(np.ascontiguousarray(sl))
+    qs, ss = oracle.quantize_act_per_token(sl)
+    assert (qd == qs).all() and (sd == ss).all()
+    assert (ss == (np.abs(bits_to_f64(np.ascontiguousarray(sl))).max(axis=1) / 127.0).astype(np.float32)).all()
 
 
 # --------------------------------------------------------------------------- integer GEMM
