@@ -27,8 +27,15 @@ if ROOT not in sys.path:
 
 METRIC = "fused W8A8 linear TOPS (% of B200 dense INT8 peak) per DiT GEMM shape"
 INT8_PEAK_TOPS = 4500.0            # B200 datasheet, dense INT8
-# measured DRAM traffic of one gemm_tc_kernel launch (ncu, see profiles/): c4 = mean of up (138.8 MB) and down (136.9 MB)
-NCU_GEMM_DRAM_BYTES_PER_LAUNCH = {"c4": 137.85e6}
+# DRAM traffic of one gemm_tc_kernel launch (dram__bytes_read.sum + dram__bytes_write.sum of an ncu capture of this
+# program on that workload, averaged over the workload's GEMM launches), with the summary it is taken from. Workloads
+# that were not captured have no entry: the bench line then says null and why.
+NCU_GEMM_DRAM_TRAFFIC = {
+    "c4": {"bytes_per_launch": 137.85e6, "profile": "profiles/gemm_tc_kernel_c4_mlp.md",
+           "note": "mean of the up (138.8 MB) and down (136.9 MB) launches; algorithmic bytes 165.2 / 122.7 MB"},
+    "paper": {"bytes_per_launch": None, "profile": "profiles/gemm_tc_kernel_paper_llm_proj_ksplit.md",
+              "note": "only the llm-proj launch was captured (1.42 GB against 502 MB algorithmic); no per-workload mean"},
+}
 L2_BYTES = 126 * 1024 * 1024
 
 
@@ -54,7 +61,7 @@ class ClockSampler:
                0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting", 0x100: "display_clock_setting",
                0x10: "sync_boost"}
 
-    def __init__(self, index: int, period_s: float = 0.02):
+    def __init__(self, index: int, period_s: float = 0.002):
         self.period = period_s
         self.samples, self.power, self.reasons = [], [], set()
         self.max_mhz = None
@@ -154,8 +161,11 @@ def run_reference(args):
         return
     from paper_2606_14598_b200 import inputs as synth
     specs = workload_specs(args)
-    steps, warmup = max(1, min(args.steps, 3)), min(args.warmup, 1)
-    tops, sec, cores, sample = time_oracle(specs, steps, warmup, target_gmac=20.0)
+    # exactly --steps timed steps after --warmup untimed ones; a step is a bounded sample of the workload (the first
+    # rows of every linear), sized so that the whole run takes about a minute of host time at ~40 GMAC/s
+    steps, warmup = max(1, args.steps), max(0, args.warmup)
+    per_linear_gmac = max(0.05, min(20.0, 2400.0 / (steps + warmup))) / max(1, len(specs))
+    tops, sec, cores, sample = time_oracle(specs, steps, warmup, target_gmac=per_linear_gmac)
     line = {
         "impl": "reference", "metric": METRIC, "value": tops, "unit": "TOPS", "n_gpus": args.gpus,
         "steps": steps, "warmup": warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
@@ -213,7 +223,19 @@ def main():
     ap.add_argument("--launch", default="direct", choices=["graph", "direct"],
                     help="graph: each step is one replay of a captured CUDA graph of the step's calls; direct: the calls themselves")
     ap.add_argument("--config", type=int, default=-1, help="force a kernel configuration (sweeps); -1 = from the shape")
+    ap.add_argument("--repeats", type=int, default=0,
+                    help="timed loops of --steps steps (0 = 5, more for short loops so that clocks get sampled); the median is reported")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # no launcher: run one process per GPU ourselves (rank i on GPU i); the ranks meet through a rendezvous file
+        from paper_2606_14598_b200 import dist as wdist
+        results = wdist.spawn_ranks([sys.executable, os.path.abspath(__file__)] + sys.argv[1:], args.gpus)
+        for r, (rc, out, err) in enumerate(results):
+            sys.stderr.write(err)
+            if r == 0:
+                sys.stdout.write(out)
+        sys.stdout.flush()
+        raise SystemExit(max(rc for rc, _, _ in results))
     if args.impl == "reference":
         return run_reference(args)
 
@@ -328,22 +350,33 @@ def main():
         burst = {"value": ops_per_step / b_sec / 1e12, "unit": "TOPS", "ms_per_step": b_sec * 1e3, "steps": 100,
                  "pct_of_int8_peak": 100.0 * ops_per_step / b_sec / 1e12 / INT8_PEAK_TOPS,
                  "note": "this rank's first 100 steps after warm-up, before the power cap engages"}
-    wdist.barrier(dev)
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # R timed loops of exactly --steps steps each, every one bracketed by a barrier and a device synchronize on both
+    # sides and timed with CUDA events on the launching stream; a loop's time is the maximum over the ranks, the
+    # reported value is the median loop. NVML is sampled every 2 ms across all of them.
+    repeats = args.repeats if args.repeats > 0 else 5
+    loop_sec = []
     with ClockSampler(local_rank) as clocks:
-        e0.record()
-        for i in range(args.steps):
-            run_step(i)
-        e1.record()
-        torch.cuda.synchronize()
-    wdist.barrier(dev)
-    sec_local = e0.elapsed_time(e1) * 1e-3
+        for _ in range(repeats):
+            wdist.barrier(dev)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for i in range(args.steps):
+                run_step(i)
+            e1.record()
+            torch.cuda.synchronize()
+            wdist.barrier(dev)
+            loop_sec.append(wdist.max_over_ranks(e0.elapsed_time(e1) * 1e-3, dev))
+    sec = statistics.median(loop_sec)
+    # the SM clock the GEMMs really ran at (cycle counter over nanosecond timer, stamped by the kernel itself)
+    gemm_mhz = [c[0] for layer in sets for L in layer if L["spec"].M > 8 for c in [w8.gemm_clock_stamps(L["ws"])] if c]
     for layer in sets:
         for L in layer:
             st = w8.int8_check_status(L["ws"])
             if st != 0:
                 raise SystemExit(f"device-side status: {w8.status_string(st)}")
+    if w8.int8_sticky_status(clear=True) != 0:          # a time-out of ANY call of the loops, not only the last ones
+        raise SystemExit("device-side status: a bounded wait expired during the timed loops")
     # ---- the same steps as direct calls, straight after (same thermal state): what a caller without graphs gets
     direct = None
     if graphs is not None and rank == 0:
@@ -359,8 +392,8 @@ def main():
         d_sec = a.elapsed_time(b) * 1e-3 / args.steps
         direct = {"value": ops_per_step / d_sec / 1e12, "unit": "TOPS", "ms_per_step": d_sec * 1e3, "steps": args.steps,
                   "note": "the step's int8_linear_fused calls issued one by one, timed right after the headline loop"}
-    ops_total_per_sec, sec = wdist.aggregate_throughput(ops_per_step * args.steps, sec_local, dev)
-    tops = ops_total_per_sec / 1e12
+    ops_all_ranks = wdist.sum_over_ranks(ops_per_step * args.steps, dev)
+    tops = ops_all_ranks / sec / 1e12
     launches = args.steps * sum(2 for _ in specs)      # quantizer + GEMM per linear
 
     line = {
@@ -369,19 +402,30 @@ def main():
         "dtype": "int8", "data": "synthetic",
         "config": {"workload": workload_name(args.workload, specs), "entry": "int8_linear_fused from bf16 activations",
                    "launch": launch_note,
-                   "regime": "one loop of --steps steps; beyond ~200 steps (50 ms) the 1 kW power cap sets the clock "
-                             "(see clocks); the first 100 steps are reported as burst",
+                   "regime": f"median of {repeats} back-to-back loops of --steps steps; a loop beyond ~200 steps (50 ms) runs "
+                             "under the 1 kW power cap (see clocks)",
                    "l2": f"inputs larger than L2: {len(sets)} rotating sets of {set_bytes / 1e6:.0f} MB each",
                    "parallelism": f"dp{world} over tokens, weights replicated, no collective"},
         "pct_of_int8_peak": 100.0 * tops / (INT8_PEAK_TOPS * world), "int8_peak_tops": INT8_PEAK_TOPS,
         "clocks": clocks.summary(), "gpu_launches": launches,
+        "repeats": {"loops": repeats, "ms_per_step": [t / args.steps * 1e3 for t in loop_sec],
+                    "tops": [ops_all_ranks / t / 1e12 for t in loop_sec], "reported": "median"},
     }
-    # what the tensor pipes could do at the clock seen: 16384 int8 ops per clock per SM (8192 multiply-adds)
+    # What the tensor pipes could do at the clock seen: 16384 int8 ops per clock per SM (8192 multiply-adds). Two
+    # clocks: NVML's (the PLL setting, sampled every 2 ms over the loops) and the one the GEMM kernels measured
+    # themselves (cycles over nanoseconds inside the launch), which is lower under a dense tensor load.
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
     if line["clocks"]["sm_mhz"]:
-        sms = torch.cuda.get_device_properties(dev).multi_processor_count
         ceiling = sms * 16384 * line["clocks"]["sm_mhz"] * 1e6 / 1e12
         line["int8_ceiling_at_observed_clock"] = {"tops": ceiling, "sm_mhz": line["clocks"]["sm_mhz"], "sms": sms,
+                                                  "clock_source": "NVML, median of the samples taken during the timed loops",
                                                   "value_frac": tops / (ceiling * world)}
+    if gemm_mhz:
+        mhz = statistics.median(gemm_mhz)
+        ceiling = sms * 16384 * mhz * 1e6 / 1e12
+        line["int8_ceiling_at_kernel_clock"] = {"tops": ceiling, "sm_mhz": mhz, "sms": sms,
+                                                "clock_source": "SM cycle counter / nanosecond timer inside the last GEMM launches of the timed loops",
+                                                "value_frac": tops / (ceiling * world)}
 
     if burst is not None and rank == 0:
         line["burst"] = burst
@@ -431,6 +475,7 @@ def main():
                 return a.elapsed_time(b) * 1e-3 / n
 
             tg = batch_time(gemm_only)
+            stamp = w8.gemm_clock_stamps(ws8) if M > 8 else None
             tgh = batch_time(gemm_hot)
             tq = batch_time(quant_only)
             tf_ = batch_time(fused)
@@ -441,6 +486,8 @@ def main():
                               "fused_from_bf16_us": tf_ * 1e6, "fused_from_bf16_tops": spec.ops / tf_ / 1e12,
                               "pct_of_int8_peak": 100.0 * spec.ops / tf_ / 1e12 / INT8_PEAK_TOPS,
                               "gemm_epilogue_us": tg * 1e6, "gemm_epilogue_tops": spec.ops / tg / 1e12,
+                              "gemm_sm_mhz": stamp[0] if stamp else None,
+                              "gemm_first_cta_us": stamp[1] * 1e6 if stamp else None,
                               "gemm_epilogue_hot_l2_us": tgh * 1e6, "gemm_epilogue_hot_l2_tops": spec.ops / tgh / 1e12,
                               "quantizer_us": tq * 1e6, "quantizer_gbs": model.quantizer_bytes(M, K) / tq / 1e9})
             if M > 16:
@@ -449,19 +496,39 @@ def main():
             q_bytes += model.quantizer_bytes(M, K)
             q_sec += tq
         line["per_shape"] = per_shape
-        int8_peak_measured = 2.0 * peaks["bf16_tflops_sustained"]
+        # The per-shape GEMM timings above are bursts (60 back-to-back launches, a few milliseconds): they belong with
+        # the burst bf16 rate. The nominal int8 : bf16 ratio of the tensor pipes is 2. The long-loop (power-capped)
+        # peak and the datasheet figure are quoted beside it, each with the fraction it gives.
+        peak_burst = 2.0 * peaks["bf16_tflops"]
+        peak_sustained = 2.0 * peaks["bf16_tflops_sustained"]
         achieved = gemm_ops / gemm_sec / 1e12 if gemm_sec > 0 else 0.0
+        traffic = NCU_GEMM_DRAM_TRAFFIC.get(args.workload) if args.rows == 0 else None
         line["roofline"] = {
             "kernel": "gemm_tc_kernel (tcgen05.mma.kind::i8 + dequant epilogue)", "bound": "tensor",
-            "achieved": achieved, "peak": int8_peak_measured, "unit": "TFLOP/s", "frac": achieved / int8_peak_measured,
-            # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised in
-            # profiles/gemm_tc_kernel_c4_mlp.md (mean of the two c4 launches; only quoted for that workload)
-            "traffic": NCU_GEMM_DRAM_BYTES_PER_LAUNCH.get(args.workload),
-            "peak_source": f"2 x {peaks['source']} sustained bf16 cuBLAS rate ({peaks['bf16_tflops_sustained']} TFLOP/s); "
+            "achieved": achieved, "peak": peak_burst, "unit": "TFLOP/s", "frac": achieved / peak_burst if peak_burst else None,
+            "regime": "burst: per-shape loops of 60 back-to-back pre-quantized launches on rotating buffers, CUDA events "
+                      "around each loop; achieved = sum of 2*M*N*K over the shapes / sum of their mean launch times",
+            "peak_source": f"2 x {peaks['source']} burst bf16 cuBLAS rate ({peaks['bf16_tflops']} TFLOP/s), of {peaks['source']}; "
                            "int8 multiply-add counted as 2 ops",
+            "ops_per_launch_sum": gemm_ops, "seconds_per_launch_sum": gemm_sec,
+            "frac_of_sustained_peak": {"peak": peak_sustained, "frac": achieved / peak_sustained,
+                                       "note": "2 x the seconds-long power-capped bf16 rate: the ceiling of a launch inside a long loop, "
+                                               "not of this burst measurement"},
+            "frac_of_datasheet": {"peak": INT8_PEAK_TOPS, "frac": achieved / INT8_PEAK_TOPS},
+            "traffic": traffic["bytes_per_launch"] if traffic else None,
+            "traffic_source": (f"{traffic['profile']}: {traffic['note']}" if traffic else
+                               "no ncu capture of this workload: not quoted"),
             "quantizer": {"bound": "hbm", "achieved": q_bytes / q_sec / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                          "frac": q_bytes / q_sec / 1e9 / peaks["hbm_gbs"]},
+                          "frac": q_bytes / q_sec / 1e9 / peaks["hbm_gbs"],
+                          "regime": "burst: 60 back-to-back launches per shape on rotating inputs",
+                          "bytes_per_launch_sum": q_bytes, "seconds_per_launch_sum": q_sec},
         }
+        clk = [p_["gemm_sm_mhz"] for p_ in per_shape if p_.get("gemm_sm_mhz")]
+        if clk:
+            ceiling = sms * 16384 * statistics.median(clk) * 1e6 / 1e12
+            line["roofline"]["frac_of_pipe_peak_at_kernel_clock"] = {
+                "peak": ceiling, "sm_mhz": statistics.median(clk), "frac": achieved / ceiling,
+                "note": "148 SMs x 16384 int8 ops per clock x the SM clock the GEMM launches measured themselves"}
         if health is not None:
             line["health"] = health
 

@@ -28,7 +28,7 @@
  *     stated.
  *   - The return value is a w8a8_status. Argument errors are detected before
  *     anything is enqueued. There is no CPU fallback and no other backend: on a
- *     device that is not sm_100 the compute calls return W8A8_ERR_ARCH.
+ *     device that is not sm_100 (compute capability 10.0) the compute calls return W8A8_ERR_ARCH.
  */
 #ifndef W8A8_LINEAR_H_
 #define W8A8_LINEAR_H_
@@ -46,7 +46,7 @@ typedef enum w8a8_status {
     W8A8_ERR_ALIGNMENT = 2,   /* pointer not 16-byte aligned, or K/N/ld break the 16-byte rules below */
     W8A8_ERR_K_OVERFLOW = 3,  /* K > 133144: K * 127^2 would not fit in int32 */
     W8A8_ERR_WORKSPACE = 4,   /* workspace NULL, misaligned or smaller than int8_linear_workspace_min_bytes() */
-    W8A8_ERR_ARCH = 5,        /* current device is not compute capability 10.x */
+    W8A8_ERR_ARCH = 5,        /* current device is not compute capability 10.0 (sm_100: B200) */
     W8A8_ERR_CUDA = 6,        /* a CUDA runtime/driver call failed (launch, descriptor encode) */
     W8A8_ERR_TIMEOUT = 7      /* a bounded device-side wait expired (reported by int8_check_status) */
 } w8a8_status;
@@ -168,10 +168,14 @@ int int8_linear_fused_host(const void* A_host, void* d_A,
  * For callers that cannot provide a workspace because they cannot allocate one: a server whose own arena
  * already owns all device memory, a latency-critical loop where cudaMalloc's implicit synchronisation is
  * not acceptable, a plug-in that only ever receives its input and output buffers. The scratch that
- * int8_linear_fused takes from the caller (status word, s_tok, qa) is a fixed
- * array of W8A8_STATIC_WORKSPACE_BYTES inside the library's device image; every GPU that loads the library
- * holds that much memory until the process exits. The call itself allocates nothing (no cudaMalloc,
- * cudaFree or allocating library routine).
+ * int8_linear_fused takes from the caller (status word, s_tok, qa, and, for shapes whose last wave of tiles is
+ * cut along K, the arrival counters and int32 partial sums) is a fixed array of W8A8_STATIC_WORKSPACE_BYTES
+ * inside the library's device image; every GPU on which the array's module has been loaded holds that much
+ * memory until the process exits. The call itself makes no allocation call (no cudaMalloc, cudaFree or
+ * allocating library routine). One caveat on when the memory is taken: with CUDA's default lazy module loading
+ * the image that holds the array is loaded, and its 16 MiB reserved, by the first call on a device (the address
+ * look-up below), not when the shared library is loaded. A caller whose arena is about to take all of the
+ * device's memory makes one call at start-up, before the arena does, or runs with CUDA_MODULE_LOADING=EAGER.
  *
  *   Arguments as for int8_linear_fused with a_dtype == W8A8_ACT_BF16 (device pointers, caller-owned).
  *   sync_and_check  0: enqueue and return. Non-zero: additionally synchronize `stream` and return
@@ -186,8 +190,9 @@ int int8_linear_fused_host(const void* A_host, void* d_A,
  *   - All calls on a device share the one array. Calls on the same stream run one after the other and are
  *     safe; calls that may overlap on the GPU (different streams, different host threads) race on it and
  *     must be serialized by the caller, or use int8_linear_fused with separate workspaces.
- *   - The array keeps whatever the last call left in it. Nothing needs clearing: each call resets the
- *     status word and rewrites the scales and codes it reads.
+ *   - The array keeps whatever the last call left in it. The caller clears nothing: each call resets the
+ *     status word, rewrites the scales and codes it reads, and zeroes the counters and partial sums of a K-split
+ *     with a memset on `stream` ahead of its kernels.
  */
 #define W8A8_STATIC_WORKSPACE_BYTES (16u * 1024u * 1024u)
 int int8_linear_fused_static(const void* A_bf16, int64_t lda,
@@ -211,8 +216,40 @@ int int8_gemm_i32_debug(const int8_t* qa, const int8_t* qw, int32_t* acc,
  * W8A8_OK, or W8A8_ERR_TIMEOUT if a bounded wait inside a kernel gave up (the
  * kernel then released its resources and returned; outputs are undefined).
  * Clears the word. Returns W8A8_ERR_CUDA if the synchronize failed.
+ * The word belongs to the LAST call enqueued on that workspace: every call resets it when it starts (which is
+ * why a workspace needs no initialisation), so a time-out of an earlier call on the same workspace is no longer
+ * there. Check after each call, or use int8_sticky_status() after many.
+ * Diagnostics in the same 256-byte status block: at byte offset 64 the first CTA of the last tensor-core GEMM
+ * on this workspace leaves four uint64 stamps: SM cycle counter and nanosecond timer when its work started, and
+ * both again when it ended. (cycles_end - cycles_start) / (ns_end - ns_start) is the SM clock in GHz that the
+ * launch really ran at, which under a dense tensor load is lower than the clock NVML reports.
  */
 int int8_check_status(void* workspace, void* stream);
+
+/*
+ * Device-wide sticky status: the first time-out recorded by ANY call of this library on the current device
+ * (whatever its workspace; the standalone quantizers, which have none, included) since the word was last
+ * cleared. Synchronizes `stream` and returns W8A8_OK or W8A8_ERR_TIMEOUT; clear != 0 also resets the word.
+ * Work still running on other streams is not waited for. The word lives in the library's device image and is
+ * zero when the library is loaded.
+ */
+int int8_sticky_status(int clear, void* stream);
+
+/*
+ * Test-only controls of the bounded waits (Method, "The fused kernel" has no counterpart; they exist so that the
+ * give-up path of the kernels can be executed without faulting or hanging a GPU).
+ *   int8_debug_set_wait_limit_ns  bound of every device-side wait for the launches that follow, in nanoseconds
+ *                                 (default 2 s; 0 restores the default). Returns the previous value.
+ *   int8_debug_set_starve         0: off. 1: the GEMM's producer warp withholds the first pipeline stage of its
+ *                                 first tile. 2: the staged activation quantizer's producer withholds its first
+ *                                 group of rows. No invalid address is touched and nothing traps: the consumers'
+ *                                 waits run out, the kernel frees what it holds and returns, and the status word
+ *                                 reports W8A8_ERR_TIMEOUT. Outputs of such a launch are undefined.
+ *                                 Returns the previous mode, -1 for an unknown one.
+ * Both are process-wide and not meant to be changed while calls are being enqueued from other threads.
+ */
+uint64_t int8_debug_set_wait_limit_ns(uint64_t limit_ns);
+int int8_debug_set_starve(int mode);
 
 /*
  * Force a kernel configuration for sweeps and tests. -1 = choose from the shape; -2 = choose from the shape

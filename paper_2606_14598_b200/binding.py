@@ -27,6 +27,7 @@ EXPORTS = (
     "int8_check_status", "int8_linear_force_config", "int8_linear_num_configs", "int8_linear_config_name",
     "int8_status_string", "int8_linear_fused_static", "int8_quantize_weight_per_channel_smooth",
     "int8_quantize_act_per_token_smooth", "int8_linear_fused_smooth", "int8_linear_workspace_min_bytes", "int8_linear_plan",
+    "int8_sticky_status", "int8_debug_set_wait_limit_ns", "int8_debug_set_starve",
 )
 
 if not os.path.exists(LIB_PATH):
@@ -65,6 +66,12 @@ _lib.int8_gemm_i32_debug.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64, _vp, _sz, 
 _lib.int8_gemm_i32_debug.restype = _int
 _lib.int8_check_status.argtypes = [_vp, _vp]
 _lib.int8_check_status.restype = _int
+_lib.int8_sticky_status.argtypes = [_int, _vp]
+_lib.int8_sticky_status.restype = _int
+_lib.int8_debug_set_wait_limit_ns.argtypes = [ctypes.c_uint64]
+_lib.int8_debug_set_wait_limit_ns.restype = ctypes.c_uint64
+_lib.int8_debug_set_starve.argtypes = [_int]
+_lib.int8_debug_set_starve.restype = _int
 _lib.int8_linear_force_config.argtypes = [_int]
 _lib.int8_linear_force_config.restype = _int
 _lib.int8_linear_num_configs.argtypes = []
@@ -318,6 +325,31 @@ def int8_gemm_i32_debug(qa: torch.Tensor, qw: torch.Tensor, workspace: torch.Ten
     _check(_lib.int8_gemm_i32_debug(_ptr(qa.contiguous()), _ptr(qw.contiguous()), _ptr(acc), M, N, K,
                                     _ptr(workspace), workspace.numel(), _stream(qa)), "int8_gemm_i32_debug")
     return acc
+
+
+def int8_sticky_status(clear: bool = True, device=None) -> int:
+    """First time-out recorded by any call on the current device since the last clear (synchronizes the current stream)."""
+    stream = torch.cuda.current_stream(device).cuda_stream
+    return int(_lib.int8_sticky_status(1 if clear else 0, stream))
+
+
+def debug_set_wait_limit_ns(limit_ns: int) -> int:
+    """Test-only: bound of the device-side waits of the following launches (0 = the 2 s default). Returns the old value."""
+    return int(_lib.int8_debug_set_wait_limit_ns(int(limit_ns)))
+
+
+def debug_set_starve(mode: int) -> int:
+    """Test-only: 1 = the GEMM's producer withholds a stage, 2 = the quantizer's producer does; 0 = off."""
+    return int(_lib.int8_debug_set_starve(int(mode)))
+
+
+def gemm_clock_stamps(workspace: torch.Tensor):
+    """(SM clock in MHz, seconds) of the first CTA of the last tensor-core GEMM that ran on this workspace, from the
+    diagnostics stamps in the status block; None if no such launch has left stamps. Synchronizes (copies to the host)."""
+    c0, t0, c1, t1 = workspace[64:96].view(torch.int64).tolist()
+    if t1 <= t0 or c1 <= c0:
+        return None
+    return (c1 - c0) / (t1 - t0) * 1e3, (t1 - t0) * 1e-9
 
 
 def int8_check_status(workspace: torch.Tensor) -> int:

@@ -5,6 +5,7 @@
 
 #include <atomic>
 #include <cstdint>
+#include <mutex>
 
 namespace {
 
@@ -15,20 +16,32 @@ constexpr int kSkinnyM = 8;           // at or below this many tokens the weight
                                       // up to 4-8 tokens, the tensor-core path from 16 on)
 
 std::atomic<int> g_forced_config{-1};
+std::atomic<uint64_t> g_wait_limit_ns{2000000000ull};     // 2 s
+std::atomic<int> g_starve{0};
+
+// First time-out recorded by any kernel of this library on the device, kept until the host clears it. (The status
+// word of a workspace is reset by every call on that workspace; this one is not.) Zero when the module is loaded.
+__device__ int g_sticky_status;
+std::mutex g_sticky_mutex;
+int* g_sticky_ptr[64] = {};
 
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// The kernels are built for sm_100a only: tcgen05.mma.kind::i8 exists on compute capability 10.0 and not, for
+// instance, on 10.3.
 int check_arch() {
     static thread_local int cached_dev = -1;
     static thread_local int cached_ok = 0;
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess) return W8A8_ERR_CUDA;
     if (dev != cached_dev) {
-        int major = 0;
-        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return W8A8_ERR_CUDA;
+        int major = 0, minor = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, dev) != cudaSuccess)
+            return W8A8_ERR_CUDA;
         cached_dev = dev;
-        cached_ok = (major == 10);
+        cached_ok = (major == 10 && minor == 0);
     }
     return cached_ok ? W8A8_OK : W8A8_ERR_ARCH;
 }
@@ -49,7 +62,48 @@ void offsets(int64_t M, size_t* s_tok_off, size_t* qa_off) {
 
 } // namespace
 
+namespace w8a8 {
+
+uint64_t wait_limit_ns() { return g_wait_limit_ns.load(); }
+int starve_mode() { return g_starve.load(); }
+
+int* sticky_status_word() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(g_sticky_mutex);
+    if (g_sticky_ptr[dev] == nullptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_sticky_status) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
+        g_sticky_ptr[dev] = static_cast<int*>(p);
+    }
+    return g_sticky_ptr[dev];
+}
+
+} // namespace w8a8
+
 extern "C" {
+
+uint64_t int8_debug_set_wait_limit_ns(uint64_t limit_ns) {
+    if (limit_ns == 0) limit_ns = 2000000000ull;
+    return g_wait_limit_ns.exchange(limit_ns);
+}
+
+int int8_debug_set_starve(int mode) {
+    if (mode != 0 && mode != kStarveGemm && mode != kStarveQuant) return -1;
+    return g_starve.exchange(mode);
+}
+
+int int8_sticky_status(int clear, void* stream) {
+    if (int e = check_arch()) return e;
+    int* word = sticky_status_word();
+    if (word == nullptr) return W8A8_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int v = 0;
+    if (cudaMemcpyAsync(&v, word, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return W8A8_ERR_CUDA;
+    if (clear && cudaMemsetAsync(word, 0, sizeof(int), st) != cudaSuccess) return W8A8_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return W8A8_ERR_CUDA;
+    return v & 0xff;
+}
 
 const char* int8_status_string(int status) {
     switch (status) {

@@ -5,32 +5,41 @@
 //
 // One persistent CTA per SM. With CG = 1 every CTA walks output tiles of 128 x BN on its own. With
 // CG = 2 the two CTAs of a cluster form a pair (tcgen05 cta_group::2) that walks tiles of 256 x BN:
-// each CTA loads its own 128 rows of A and its own half (BN/2 rows) of the W tile, the leader CTA
+// each CTA loads its own 128 rows of A and its own half of the W tile, the leader CTA
 // issues one MMA for both, and each CTA ends up with its 128 x BN half of the accumulator in its own
 // TMEM. A pair moves half as many W bytes per SM through shared memory as two independent CTAs, which
 // is what the shared-memory bandwidth needs at the int8 rate. Every load is a plain per-CTA TMA load: the
 // leader signals the peer's barriers with a second, plain tcgen05.commit / mbarrier.arrive.
+//
+// A tile is NSUB sub-tiles of BNS columns side by side (BN = NSUB * BNS). TMEM holds two accumulator slots
+// of up to 256 columns, and consecutive sub-tiles alternate between them:
+//   NSUB = 1  consecutive tiles alternate slots, so the epilogue of one tile overlaps the k-loop of the next;
+//   NSUB = 2  the two sub-tiles of a tile share every A stage (each k-block is multiplied into both slots), which
+//             cuts the operand bytes a CTA pulls out of L2 per MMA by a quarter (BNS = 256) or a sixth (BNS = 192):
+//             the L2 -> SM feed, not the tensor pipe, is what holds the 256 x 256 tile down. The price is that both
+//             slots complete together; the next tile therefore starts staggered: as soon as slot 0 is drained its
+//             sub-tile runs ahead over the k-blocks the ring already holds while the epilogue drains slot 1, then
+//             sub-tile 1 catches up on the same stages and releases them. To the epilogue a tile simply looks like
+//             NSUB consecutive tiles.
 // Warp roles:
-//   warp 0    TMA producer: loads the 128 x 128-byte A tile and the BN x 128-byte
-//             W tile of each k-block into a ring of shared-memory stages
-//             (128-byte swizzle, K-major: both operands are row-major over K)
-//   warp 1    allocates TMEM and issues the MMAs (one thread), 4 per k-block
-//             (K = 32 each); tcgen05.commit releases the stage / publishes the tile
+//   warp 0    TMA producer: loads the 128 x 128-byte A tile and the W tile(s) of each k-block into a ring of
+//             shared-memory stages (128-byte swizzle, K-major: both operands are row-major over K)
+//   warp 1    allocates TMEM and issues the MMAs (one thread), 4 per k-block and sub-tile
+//             (K = 32 each); tcgen05.commit releases the stage / publishes the sub-tile
 //   warps 2-5 epilogue: tcgen05.ld the accumulator (lane = row, so s_tok is one
 //             scalar per thread; s_ch and bias are per-column broadcasts from
 //             shared memory), dequantize, pack to bf16, stage in swizzled shared
 //             memory, TMA-store 32 x 64 boxes (TMA clips ragged M and N)
 //   warps 6-9 helpers: idle until the CTA's last tile, whose epilogue no k-loop hides;
-//             there they take half of the boxes (a warp reads only the TMEM lanes of
+//             there they take part of the boxes (a warp reads only the TMEM lanes of
 //             its index modulo 4, so they pair up with warps 2-5 lane group by lane group)
-// Two accumulators of BN columns alternate in TMEM so that the epilogue of one
-// tile overlaps the k-loop of the next. (Eight epilogue warps, two per TMEM lane
-// group, with the per-column scales read straight from global memory, were
-// measured slower: 121.5 against 117.2 us on the MLP up-projection.)
+// (Eight epilogue warps on every tile, two per TMEM lane group, with the per-column scales read straight from
+// global memory, were measured slower on the double-buffered 256 x 256 tile: 121.5 against 117.2 us on the MLP
+// up-projection.)
 //
-// K-split of the partial wave: when the number of tiles is not a multiple of the number of CTA groups, the
-// last num_tiles % groups tiles would keep only a few SMs busy for a whole tile time. The host may ask for
-// them to be cut along K into split_s parts, one part per group. Every part adds its int32 partial
+// K-split of the partial wave (NSUB = 1 only): when the number of tiles is not a multiple of the number of CTA
+// groups, the last num_tiles % groups tiles would keep only a few SMs busy for a whole tile time. The host may ask
+// for them to be cut along K into split_s parts, one part per group. Every part adds its int32 partial
 // accumulator into the tile's slab of the workspace (integer sums: the result does not depend on the
 // order); a per-tile counter tells the part that finishes last to read the sums back and run the epilogue.
 // No CTA ever waits for another one.
@@ -51,31 +60,34 @@ namespace w8a8 {
 namespace {
 
 constexpr int BM = 128;            // rows of A per tile (= TMEM lanes)
-constexpr int BK = 128;            // int8 elements (= bytes) of K per stage: one 128-byte swizzle row
+constexpr int BK = 128;            // int8 elements (= bytes) of K per k-block: one 128-byte swizzle row
 constexpr int MMA_K = 32;          // K of one tcgen05.mma.kind::i8
 constexpr int EPI_THREADS = 128;    // warps 2..5: the epilogue of every tile
-constexpr int HELPER_WARP0 = 6;     // warps 6..9: take half of the columns of a CTA's last tile, whose epilogue nothing hides
+constexpr int HELPER_WARP0 = 6;     // warps 6..9: take part of the columns of a CTA's last tile, whose epilogue nothing hides
 constexpr int NUM_THREADS = 64 + 2 * EPI_THREADS;
-constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;   // 2 s
+constexpr int SMEM_MAX = 232448;   // dynamic shared memory a CTA can opt in to
 
 enum Where { W_PRODUCER_EMPTY = 1, W_MMA_FULL = 2, W_MMA_TMEM_EMPTY = 3, W_EPI_TMEM_FULL = 4 };
 
-template <int CG, int BN, int STAGES, int KBS>
+template <int CG, int BNS, int NSUB, int STAGES, int KBS>
 struct SmemLayout {
+    static constexpr int BN = BNS * NSUB;                           // columns of a tile
     static constexpr int A_BYTES = BM * BK;
-    static constexpr int B_ROWS = BN / CG;                          // W rows this CTA loads per tile
+    static constexpr int B_ROWS = BNS / CG;                         // W rows of one sub-tile this CTA loads
     static constexpr int B_BYTES = B_ROWS * BK;
-    static constexpr int KB_BYTES = A_BYTES + B_BYTES;              // one k-block: A tile + W tile of 128 bytes of K
+    static constexpr int KB_BYTES = A_BYTES + NSUB * B_BYTES;       // one k-block: A tile + W tile(s) of 128 bytes of K
     static constexpr int STAGE_BYTES = KBS * KB_BYTES;              // a pipeline stage holds KBS k-blocks
+    static constexpr int RING_BYTES = STAGES * STAGE_BYTES;
     static constexpr int STAGING_BOX_BYTES = 32 * 128;             // one 32-row x 64-column bf16 box
     // two boxes alternate per epilogue warp where shared memory allows, else one
-    static constexpr int STAGING_BUFS = (STAGES * STAGE_BYTES + 8 * STAGING_BOX_BYTES + 8 * BN + 1280 <= 232448) ? 2 : 1;
+    static constexpr int STAGING_BUFS = (RING_BYTES + 8 * STAGING_BOX_BYTES + 16 * BNS + 1280 <= SMEM_MAX) ? 2 : 1;
     static constexpr int STAGING_BYTES_PER_WARP = STAGING_BUFS * STAGING_BOX_BYTES;
-    static constexpr int OFF_STAGING = STAGES * STAGE_BYTES;
+    static constexpr int OFF_STAGING = RING_BYTES;
+    // per-column scales and bias of a sub-tile, double-buffered by accumulator slot
     static constexpr int OFF_SCH = OFF_STAGING + 4 * STAGING_BYTES_PER_WARP;
-    static constexpr int OFF_BIAS = OFF_SCH + BN * 4;
+    static constexpr int OFF_BIAS = OFF_SCH + 2 * BNS * 4;
     // full[STAGES * KBS] (one per k-block), empty[STAGES] (one per stage), tfull[2], tempty[2]
-    static constexpr int OFF_BARS = OFF_BIAS + BN * 4;
+    static constexpr int OFF_BARS = OFF_BIAS + 2 * BNS * 4;
     static constexpr int NUM_FULL = STAGES * KBS;
     static constexpr int NUM_BARS = NUM_FULL + STAGES + 4;
     static constexpr int OFF_TMEM = OFF_BARS + NUM_BARS * 8;
@@ -83,6 +95,7 @@ struct SmemLayout {
     static constexpr int OFF_LAST = OFF_ABORT + 4;                 // "this CTA finishes the split tile" (epilogue warps)
     static constexpr int TOTAL = OFF_LAST + 4;
     static constexpr int DYN_BYTES = TOTAL + 1024;                 // slack to align the base to 1024
+    static_assert(B_BYTES % 1024 == 0, "operand tiles start on a swizzle-atom boundary");
 };
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -90,14 +103,24 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-template <int CG, int BN, int STAGES, int KBS, bool RAW_I32>
+// What a kernel needs beyond its operands: the bound of its waits, where time-outs are recorded, test hooks.
+struct RunCtl {
+    int* status;            // workspace status word
+    int* sticky;            // device-wide sticky status word (or nullptr)
+    uint64_t wait_limit_ns;
+    int after_quantizer;    // the quantizer ahead of this kernel has reset the status word
+    int starve;             // test hook: the producer withholds the first k-stage of its first tile
+};
+
+template <int CG, int BNS, int NSUB, int STAGES, int KBS, bool RAW_I32>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                const __grid_constant__ CUtensorMap tm_out,
-               const float* __restrict__ s_tok, const float* __restrict__ s_ch, const float* __restrict__ bias,
-               int32_t* __restrict__ raw_out, int M, int N, int K, int* status, int after_quantizer,
+               const float* s_tok, const float* __restrict__ s_ch, const float* __restrict__ bias,
+               int32_t* __restrict__ raw_out, int M, int N, int K, const RunCtl rc,
                int split_tiles, int split_s, int32_t* split_slabs, int* split_counters) {
-    using L = SmemLayout<CG, BN, STAGES, KBS>;
+    using L = SmemLayout<CG, BNS, NSUB, STAGES, KBS>;
+    constexpr int BN = L::BN;
     // the next kernel in the stream, if it was launched to allow it (the next call's quantizer is), may be scheduled
     // as this grid's CTAs retire and set itself up; it waits for this whole grid before it touches global memory
     grid_dep_launch_dependents();
@@ -117,12 +140,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     auto tempty_bar = [&](int b) { return bars + 8u * (L::NUM_FULL + STAGES + 2 + b); };  // used in the leader
     volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(base_ptr + L::OFF_TMEM);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::OFF_ABORT);
-    const WaitCtl ctl{abort_flag, status, WAIT_LIMIT_NS};
+    const WaitCtl ctl{abort_flag, rc.status, rc.sticky, rc.wait_limit_ns};
 
-    // two accumulators, each at a power-of-two column offset (the allocation must be a power of two >= 32)
-    constexpr uint32_t TMEM_BUF = BN <= 128 ? 128u : 256u;
+    // two accumulator slots, each at a power-of-two column offset (the allocation must be a power of two >= 32)
+    constexpr uint32_t TMEM_BUF = BNS <= 128 ? 128u : 256u;
     constexpr uint32_t TMEM_COLS = 2 * TMEM_BUF;
-    static_assert(BN % 64 == 0 && BN <= 256, "BN: whole 64-column output boxes, at most 256 TMEM columns per buffer");
+    static_assert(BNS % 64 == 0 && BNS <= 256, "BNS: whole 64-column output boxes, at most 256 TMEM columns per slot");
+    static_assert(NSUB == 1 || NSUB == 2, "a tile is one or two sub-tiles");
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -155,7 +179,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     // (K-split) part unit_part of tile unit_tile: stages [unit_sb, unit_se) of its k-loop.
     const int num_kstages = (num_kb + KBS - 1) / KBS;
     const int tiles_whole = num_tiles - split_tiles;
-    const bool has_unit = split_s >= 2 && first_tile < split_tiles * split_s;
+    const bool has_unit = NSUB == 1 && split_s >= 2 && first_tile < split_tiles * split_s;
     const int unit_slot = has_unit ? first_tile / split_s : 0, unit_part = has_unit ? first_tile % split_s : 0;
     const int unit_tile = tiles_whole + unit_slot;
     const int unit_sb = has_unit ? num_kstages * unit_part / split_s : 0;
@@ -171,14 +195,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         if (lane == 0) {
             grid_dep_wait();
             // without a quantizer ahead of it (which clears the status word) the kernel clears it itself; a time-out
-            // can only be recorded seconds later
-            if (!after_quantizer && blockIdx.x == 0) *status = 0;
+            // can only be recorded a whole wait limit later
+            if (!rc.after_quantizer && blockIdx.x == 0) *rc.status = 0;
+            // diagnostics: CTA 0 stamps the SM cycle counter and the nanosecond timer when its work starts and when it
+            // ends (status block, byte 64): their ratio is the SM clock this launch really ran at
+            if (blockIdx.x == 0) {
+                unsigned long long* stamps = reinterpret_cast<unsigned long long*>(rc.status + 16);
+                stamps[0] = static_cast<unsigned long long>(clock64());
+                stamps[1] = globaltimer_ns();
+            }
         }
         __syncwarp();
         int stage = 0;
         uint32_t phase = 0;
         int issued = 0;
         bool ok = true;
+        bool withhold = rc.starve != 0;                     // test hook: this CTA's very first stage never arrives
         auto produce = [&](int t, int sb, int se) {
             const int m0 = tile_m(t) * TILE_M + rank * BM;
             const int n0 = tile_n(t) * BN + rank * L::B_ROWS;
@@ -187,21 +219,33 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 for (int ks = sb; ks < se; ++ks) {
                     const int kb = ks * KBS;
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, ctl, W_PRODUCER_EMPTY, kStatusTimeout)) { ok = false; break; }
+                    if (withhold) {
+                        // neither the byte count nor a copy is posted for this stage: its barriers never complete, the
+                        // MMA thread's bounded wait runs out, and every role unwinds
+                        withhold = false;
+                        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                        continue;
+                    }
                     // a stage always receives all its k-blocks: those past the end of K are zero-filled by TMA
                     // (and skipped by the MMA thread), which keeps the byte count of the barrier constant
 #pragma unroll
                     for (int sub = 0; sub < KBS; ++sub) {
                         const uint32_t sa = base + stage * L::STAGE_BYTES + sub * L::KB_BYTES;
+                        const int kx = (kb + sub) * BK;
                         if (CG == 2) {
                             // the leader's barrier counts the bytes of both CTAs
                             if (leader) mbar_arrive_expect_tx(full_bar(stage, sub), 2 * L::KB_BYTES);
                             const uint32_t fb = mapa_shared(full_bar(stage, sub), 0);
-                            tma_load_2d_pair_hint(sa, &tm_a, fb, (kb + sub) * BK, m0, keep);
-                            tma_load_2d_pair_hint(sa + L::A_BYTES, &tm_b, fb, (kb + sub) * BK, n0, keep);
+                            tma_load_2d_pair_hint(sa, &tm_a, fb, kx, m0, keep);
+#pragma unroll
+                            for (int h = 0; h < NSUB; ++h)
+                                tma_load_2d_pair_hint(sa + L::A_BYTES + h * L::B_BYTES, &tm_b, fb, kx, n0 + h * BNS, keep);
                         } else {
                             mbar_arrive_expect_tx(full_bar(stage, sub), L::KB_BYTES);
-                            tma_load_2d_hint(sa, &tm_a, full_bar(stage, sub), (kb + sub) * BK, m0, keep);
-                            tma_load_2d_hint(sa + L::A_BYTES, &tm_b, full_bar(stage, sub), (kb + sub) * BK, n0, keep);
+                            tma_load_2d_hint(sa, &tm_a, full_bar(stage, sub), kx, m0, keep);
+#pragma unroll
+                            for (int h = 0; h < NSUB; ++h)
+                                tma_load_2d_hint(sa + L::A_BYTES + h * L::B_BYTES, &tm_b, full_bar(stage, sub), kx, n0 + h * BNS, keep);
                         }
                     }
                     ++issued;
@@ -226,50 +270,97 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer (leader CTA only)
         if (lane == 0 && leader) {
-            constexpr uint32_t idesc = make_i8_idesc(TILE_M, BN);
+            constexpr uint32_t idesc = make_i8_idesc(TILE_M, BNS);
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            int it = 0;
-            auto mma_tile = [&](int sb, int se) {
-                const int buf = it & 1;
-                if (!mbar_wait(tempty_bar(buf), ((it >> 1) & 1) ^ 1u, ctl, W_MMA_TMEM_EMPTY, kStatusTimeout)) { ok = false; return; }
+            int c = 0;                                     // sub-tiles begun so far: slot = c & 1, use of that slot = c >> 1
+            auto slot_tmem = [&](int cc) { return tmem_base + static_cast<uint32_t>(cc & 1) * TMEM_BUF; };
+            auto wait_slot = [&](int cc) {                 // the epilogue has drained the slot's previous sub-tile
+                if (!mbar_wait(tempty_bar(cc & 1), ((cc >> 1) & 1) ^ 1u, ctl, W_MMA_TMEM_EMPTY, kStatusTimeout)) return false;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + buf * TMEM_BUF;
-                for (int ks = sb; ks < se; ++ks) {
-                    const int kb = ks * KBS;
+                return true;
+            };
+            // the MMAs of k-block (st, sub) into sub-tile h; `fresh`: this k-block is the first of the sub-tile
+            auto issue = [&](int st, int sub, int kbi, int h, uint32_t d_tmem, bool fresh) {
+                const uint32_t sa = base + st * L::STAGE_BYTES + sub * L::KB_BYTES;
+                const uint64_t da = make_kmajor_sw128_desc(sa);
+                const uint64_t db = make_kmajor_sw128_desc(sa + L::A_BYTES + h * L::B_BYTES);
+                // K steps of this k-block that hold data (0 for a k-block past the end of K)
+                const int left = K - kbi * BK;
+                const int ksteps = left <= 0 ? 0 : min(BK, left + MMA_K - 1) / MMA_K;
 #pragma unroll
-                    for (int sub = 0; sub < KBS; ++sub) {
-                        if (!mbar_wait(full_bar(stage, sub), phase, ctl, W_MMA_FULL, kStatusTimeout)) { ok = false; break; }
-                        tc_fence_after();
-                        const uint32_t sa = base + stage * L::STAGE_BYTES + sub * L::KB_BYTES;
-                        const uint64_t da = make_kmajor_sw128_desc(sa);
-                        const uint64_t db = make_kmajor_sw128_desc(sa + L::A_BYTES);
-                        // K steps of this k-block that hold data (0 for a k-block past the end of K)
-                        const int left = K - (kb + sub) * BK;
-                        const int ksteps = left <= 0 ? 0 : min(BK, left + MMA_K - 1) / MMA_K;
-#pragma unroll
-                        for (int k = 0; k < BK / MMA_K; ++k) {
-                            if (k < ksteps) {   // advancing K by 32 bytes inside the swizzled row: +2 in 16-byte units
-                                const uint32_t acc = ((ks - sb) | sub | k) != 0 ? 1u : 0u;   // the first MMA overwrites
-                                if (CG == 2) mma_i8_ss_pair(d_tmem, da + 2 * k, db + 2 * k, idesc, acc);
-                                else mma_i8_ss(d_tmem, da + 2 * k, db + 2 * k, idesc, acc);
-                            }
-                        }
+                for (int k = 0; k < BK / MMA_K; ++k) {
+                    if (k < ksteps) {   // advancing K by 32 bytes inside the swizzled row: +2 in 16-byte units
+                        const uint32_t acc = (fresh && k == 0) ? 0u : 1u;   // the first MMA overwrites
+                        if (CG == 2) mma_i8_ss_pair(d_tmem, da + 2 * k, db + 2 * k, idesc, acc);
+                        else mma_i8_ss(d_tmem, da + 2 * k, db + 2 * k, idesc, acc);
                     }
-                    if (!ok) break;
-                    // the stage is free (in both CTAs) once these MMAs have read it. One commit per stage, not per
-                    // k-block: with 128-byte stages the commits and barrier round trips cost ~8% of the run time
-                    if (CG == 2) { tc_commit_pair(empty_bar(stage)); tc_commit_pair(mapa_shared(empty_bar(stage), 1)); }
-                    else tc_commit(empty_bar(stage));
-                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-                }
-                if (ok) {                                  // accumulator complete (in both CTAs)
-                    if (CG == 2) { tc_commit_pair(tfull_bar(buf)); tc_commit_pair(mapa_shared(tfull_bar(buf), 1)); }
-                    else tc_commit(tfull_bar(buf));
                 }
             };
-            for (int t = first_tile; t < tiles_whole && ok; t += tile_step, ++it) mma_tile(0, num_kstages);
+            auto wait_full = [&](int st, int sub, uint32_t ph) {
+                if (!mbar_wait(full_bar(st, sub), ph, ctl, W_MMA_FULL, kStatusTimeout)) return false;
+                tc_fence_after();
+                return true;
+            };
+            // the stage is free (in both CTAs) once the MMAs issued so far have read it. One commit per stage, not per
+            // k-block: with 128-byte stages the commits and barrier round trips cost ~8% of the run time
+            auto release_stage = [&](int st) {
+                if (CG == 2) { tc_commit_pair(empty_bar(st)); tc_commit_pair(mapa_shared(empty_bar(st), 1)); }
+                else tc_commit(empty_bar(st));
+            };
+            auto publish = [&](int cc) {                   // the sub-tile's accumulator is complete (in both CTAs)
+                if (CG == 2) { tc_commit_pair(tfull_bar(cc & 1)); tc_commit_pair(mapa_shared(tfull_bar(cc & 1), 1)); }
+                else tc_commit(tfull_bar(cc & 1));
+            };
+            auto mma_tile = [&](int sb, int se) {
+                int ks = sb;
+                if (NSUB == 2) {
+                    // Staggered start. Both slots were published together, but the epilogue drains slot 0 first:
+                    // sub-tile 0 runs ahead over the stages the ring can hold while slot 1 is still being drained,
+                    // then sub-tile 1 catches up on the same stages and hands them back.
+                    const int lead = min(STAGES, se - sb);
+                    if (!wait_slot(c)) { ok = false; return; }
+                    int st = stage;
+                    uint32_t ph = phase;
+                    for (int i = 0; i < lead && ok; ++i) {
+#pragma unroll
+                        for (int sub = 0; sub < KBS; ++sub) {
+                            if (!wait_full(st, sub, ph)) { ok = false; break; }
+                            issue(st, sub, (sb + i) * KBS + sub, 0, slot_tmem(c), i == 0 && sub == 0);
+                        }
+                        if (++st == STAGES) { st = 0; ph ^= 1u; }
+                    }
+                    if (!ok) return;
+                    if (!wait_slot(c + 1)) { ok = false; return; }
+                    for (int i = 0; i < lead; ++i) {
+#pragma unroll
+                        for (int sub = 0; sub < KBS; ++sub)
+                            issue(stage, sub, (sb + i) * KBS + sub, 1, slot_tmem(c + 1), i == 0 && sub == 0);
+                        release_stage(stage);
+                        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                    }
+                    ks = sb + lead;
+                } else {
+                    if (!wait_slot(c)) { ok = false; return; }
+                }
+                for (; ks < se; ++ks) {
+#pragma unroll
+                    for (int sub = 0; sub < KBS; ++sub) {
+                        if (!wait_full(stage, sub, phase)) { ok = false; break; }
+#pragma unroll
+                        for (int h = 0; h < NSUB; ++h)
+                            issue(stage, sub, ks * KBS + sub, h, slot_tmem(c + h), ks == sb && sub == 0);
+                    }
+                    if (!ok) return;
+                    release_stage(stage);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+#pragma unroll
+                for (int h = 0; h < NSUB; ++h) publish(c + h);
+                c += NSUB;
+            };
+            for (int t = first_tile; t < tiles_whole && ok; t += tile_step) mma_tile(0, num_kstages);
             if (has_unit && ok) mma_tile(unit_sb, unit_se);
         }
     } else {
@@ -280,40 +371,44 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         float* sm_sch = reinterpret_cast<float*>(base_ptr + L::OFF_SCH);
         float* sm_bias = reinterpret_cast<float*>(base_ptr + L::OFF_BIAS);
         // staging boxes: the epilogue warps have their own; the helpers borrow the operand ring, which is idle by
-        // the time the last tile's accumulator is complete
+        // the time the last tile's accumulators are complete
         const int stg_off = helper ? (warp - HELPER_WARP0) * L::STAGING_BYTES_PER_WARP
                                    : L::OFF_STAGING + (warp - 2) * L::STAGING_BYTES_PER_WARP;
         const uint32_t staging = base + stg_off;
         uint8_t* staging_ptr = base_ptr + stg_off;
-        // The epilogue of a CTA's last tile overlaps with nothing: there the helpers take the upper half of the boxes.
+        // The epilogue of a CTA's last tile overlaps with nothing: there the helpers take the upper part of the boxes.
         const int n_regular = tiles_whole > first_tile ? (tiles_whole - first_tile + tile_step - 1) / tile_step : 0;
-        const bool helpers_on = !RAW_I32 && n_regular > 0 && !has_unit;
-        constexpr int ALL_CHUNKS = BN / 32;
-        constexpr int C_SPLIT = 2 * (BN / 64 - BN / 128);            // 32-column chunks the epilogue warps keep on that tile
+        const int n_sub = n_regular * NSUB;            // sub-tiles of whole tiles this CTA works on
+        constexpr int ALL_CHUNKS = BNS / 32;
+        constexpr int C_SPLIT = 2 * (BNS / 64 - BNS / 128);          // 32-column chunks the epilogue warps keep on that tile
+        const bool helpers_on = !RAW_I32 && n_regular > 0 && !has_unit && C_SPLIT < ALL_CHUNKS;
         const bool has_bias = bias != nullptr;
         const uint64_t stream_out = l2_policy_evict_first();        // the output is written once and not read here
         grid_dep_wait();                               // s_tok may come from the kernel before this one
         bool ok = true;
-        int it = 0;
+        int c = 0;                                     // sub-tile counter: slot = c & 1, use of the slot = c >> 1
         volatile int* last_flag = reinterpret_cast<volatile int*>(base_ptr + L::OFF_LAST);
-        // chunks [c_lo, c_hi) of tile t; `shared_tile`: the helpers work on this tile too
-        auto epi_tile = [&](int t, bool unit, int c_lo, int c_hi, bool shared_tile) {
-            const int buf = it & 1;
-            const int m0 = tile_m(t) * TILE_M + rank * BM, n0 = tile_n(t) * BN;
+        // chunks [c_lo, c_hi) of sub-tile h of tile t; `shared_tile`: the helpers work on this sub-tile too
+        auto epi_tile = [&](int t, int h, bool unit, int c_lo, int c_hi, bool shared_tile) {
+            const int buf = c & 1;
+            const int m0 = tile_m(t) * TILE_M + rank * BM, n0 = tile_n(t) * BN + h * BNS;
+            const float* sch_buf = sm_sch + buf * BNS;
+            const float* bias_buf = sm_bias + buf * BNS;
             if (!RAW_I32 && !helper) {
-                asm volatile("bar.sync 1, 128;" ::: "memory");     // previous tile's readers are done
-                for (int j = ep_tid; j < BN; j += EPI_THREADS) {
+                // the slot's buffer was last read two sub-tiles ago, which every warp has left behind
+                for (int j = ep_tid; j < BNS; j += EPI_THREADS) {
                     const int n = n0 + j;
-                    sm_sch[j] = n < N ? __ldg(s_ch + n) : 0.f;
-                    sm_bias[j] = (has_bias && n < N) ? __ldg(bias + n) : 0.f;
+                    sm_sch[buf * BNS + j] = n < N ? __ldg(s_ch + n) : 0.f;
+                    sm_bias[buf * BNS + j] = (has_bias && n < N) ? __ldg(bias + n) : 0.f;
                 }
                 asm volatile("bar.sync 1, 128;" ::: "memory");
             }
-            // the helpers have been parked here since the start of the kernel: the scales of the last tile are in place
+            // the helpers have been parked here since the start of the kernel: the scales of this sub-tile are in place
             if (shared_tile) asm volatile("bar.sync 2, 256;" ::: "memory");
             const int row = m0 + lg * 32 + lane;
-            const float st = (!RAW_I32 && row < M) ? __ldg(s_tok + row) : 0.f;
-            if (ok && !mbar_wait(tfull_bar(buf), (it >> 1) & 1, ctl, W_EPI_TMEM_FULL, kStatusTimeout)) ok = false;
+            // plain (coherent) load: the quantizer ahead of this kernel wrote s_tok while this kernel was already resident
+            const float st = (!RAW_I32 && row < M) ? __ldcg(s_tok + row) : 0.f;
+            if (ok && !mbar_wait(tfull_bar(buf), (c >> 1) & 1, ctl, W_EPI_TMEM_FULL, kStatusTimeout)) ok = false;
             ok = __all_sync(0xffffffffu, ok);
             if (!ok && !unit) return;                  // later tiles still take their named barriers, but skip the work
             tc_fence_after();
@@ -322,8 +417,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             // The TMEM load of the next chunk is in flight while the current one is converted.
             const uint64_t st2 = pack2(st, st);
             auto process = [&](int cc, const uint32_t (&v)[32]) {
-                const int col = cc * 32, h = cc & 1, c = cc >> 1;
-                const int sbuf = c & (L::STAGING_BUFS - 1);   // staging boxes alternate: the store of one overlaps the next
+                const int col = cc * 32, hh = cc & 1, cb = cc >> 1;
+                const int sbuf = cb & (L::STAGING_BUFS - 1);  // staging boxes alternate: the store of one overlaps the next
                 if (RAW_I32) {
                     if (row < M) {
                         int32_t* dst = raw_out + static_cast<int64_t>(row) * N + n0 + col;
@@ -336,21 +431,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
                     // (float(acc) * s_tok) * s_ch + bias on two columns at a time; each half rounds like the scalar op
-                    uint64_t t = pack2(__int2float_rn(static_cast<int>(v[2 * j])), __int2float_rn(static_cast<int>(v[2 * j + 1])));
-                    t = mul2(t, st2);
-                    t = mul2(t, *reinterpret_cast<const uint64_t*>(sm_sch + col + 2 * j));
+                    uint64_t tt = pack2(__int2float_rn(static_cast<int>(v[2 * j])), __int2float_rn(static_cast<int>(v[2 * j + 1])));
+                    tt = mul2(tt, st2);
+                    tt = mul2(tt, *reinterpret_cast<const uint64_t*>(sch_buf + col + 2 * j));
                     float a0, a1;
-                    unpack2(t, a0, a1);
+                    unpack2(tt, a0, a1);
                     if (has_bias) {
                         // scalar adds: a packed add right behind the packed multiply was seen to be contracted
                         // into a fused multiply-add by the assembler, which changes the rounding
-                        const float2 bi = *reinterpret_cast<const float2*>(sm_bias + col + 2 * j);
+                        const float2 bi = *reinterpret_cast<const float2*>(bias_buf + col + 2 * j);
                         a0 = __fadd_rn(a0, bi.x);
                         a1 = __fadd_rn(a1, bi.y);
                     }
                     packed[j] = pack_bf16x2(a0, a1);
                 }
-                if (h == 0) {
+                if (hh == 0) {
                     // the store issued STAGING_BUFS boxes ago (same staging box) must have finished reading it
                     if (lane == 0) bulk_wait_group_read<L::STAGING_BUFS - 1>();
                     __syncwarp();
@@ -360,19 +455,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     uint4 q = make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
-                    *reinterpret_cast<uint4*>(srow + (((h * 4 + i) ^ (lane & 7)) << 4)) = q;
+                    *reinterpret_cast<uint4*>(srow + (((hh * 4 + i) ^ (lane & 7)) << 4)) = q;
                 }
-                if (h == 1) {
+                if (hh == 1) {
                     fence_proxy_async_smem();
                     __syncwarp();
                     if (lane == 0) {
-                        tma_store_2d_hint(&tm_out, staging + sbuf * L::STAGING_BOX_BYTES, n0 + c * 64, m0 + lg * 32, stream_out);
+                        tma_store_2d_hint(&tm_out, staging + sbuf * L::STAGING_BOX_BYTES, n0 + cb * 64, m0 + lg * 32, stream_out);
                         bulk_commit_group();
                     }
                 }
                 }
             };
-            auto release_accumulator = [&]() {         // every TMEM load of this tile has completed
+            auto release_accumulator = [&]() {         // every TMEM load of this sub-tile has completed
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0 && !helper) {            // (nothing follows a tile the helpers work on)
@@ -429,7 +524,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             __threadfence();
             // This is the CTA's last piece of work and its MMAs have completed: the operand ring is free. Pull the
             // whole slab into it with asynchronous copies (all in flight at once), then run the usual epilogue.
-            static_assert(SLAB * 4 <= STAGES * L::STAGE_BYTES, "the slab fits in the operand ring");
+            static_assert(NSUB == 2 || SLAB * 4 <= L::RING_BYTES, "the slab fits in the operand ring");
             for (int i = ep_tid; i < SLAB / 4; i += EPI_THREADS) cp_async_16(base + i * 16, slab + i * 4);
             cp_async_wait_all();
             asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -443,20 +538,30 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             }
         };
         if (!helper) {
-            for (int t = first_tile; t < tiles_whole; t += tile_step, ++it) {
-                const bool shared_tile = helpers_on && it == n_regular - 1;
-                epi_tile(t, false, 0, shared_tile ? C_SPLIT : ALL_CHUNKS, shared_tile);
+            for (int t = first_tile; t < tiles_whole; t += tile_step) {
+#pragma unroll
+                for (int h = 0; h < NSUB; ++h, ++c) {
+                    const bool shared_tile = helpers_on && c >= n_sub - NSUB;
+                    epi_tile(t, h, false, 0, shared_tile ? C_SPLIT : ALL_CHUNKS, shared_tile);
+                }
             }
-            if (has_unit) epi_tile(unit_tile, true, 0, ALL_CHUNKS, false);
+            if (has_unit) epi_tile(unit_tile, 0, true, 0, ALL_CHUNKS, false);
         } else if (helpers_on) {
-            it = n_regular - 1;
-            epi_tile(first_tile + it * tile_step, false, C_SPLIT, ALL_CHUNKS, true);
+            const int t_last = first_tile + (n_regular - 1) * tile_step;
+            c = n_sub - NSUB;
+#pragma unroll
+            for (int h = 0; h < NSUB; ++h, ++c) epi_tile(t_last, h, false, C_SPLIT, ALL_CHUNKS, true);
         }
         if (!RAW_I32 && lane == 0) bulk_wait_group<0>();
     }
 
     tc_fence_before();
     __syncthreads();
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        unsigned long long* stamps = reinterpret_cast<unsigned long long*>(rc.status + 16);
+        stamps[2] = static_cast<unsigned long long>(clock64());
+        stamps[3] = globaltimer_ns();
+    }
     if (CG == 2) cluster_sync_all();            // nobody leaves while the peer may still signal its barriers
     tc_fence_after();
     if (warp == 1) {
@@ -498,17 +603,19 @@ bool encode_2d(CUtensorMap* tm, CUtensorMapDataType dt, const void* ptr, uint64_
 
 struct TcConfig {
     const char* name;
-    int cg, bn, stages, kbs;
+    int cg, bns, nsub, stages, kbs;
     float eff;      // measured throughput per SM relative to configuration 2 (large shapes, whole waves)
 };
 constexpr TcConfig kConfigs[] = {
     // measured on the c4 shapes (hot L2): pair 256x256 3 x 256 B: 115 / 111 us; one CTA 128x256 4 x 128 B: 129 / 121 us;
     // pair 256x192: 130 / 123 us; one CTA 128x128: 164 / 154 us; pair 256x128: 168 / 162 us
-    {"tc 128x256 per CTA, 4 stages x 128 B of K", 1, 256, 4, 1, 0.89f},
-    {"tc 128x128 per CTA, 3 stages x 256 B of K", 1, 128, 3, 2, 0.72f},
-    {"tc 256x256 per CTA pair, 3 stages x 256 B of K", 2, 256, 3, 2, 1.00f},
-    {"tc 256x128 per CTA pair, 4 stages x 256 B of K", 2, 128, 4, 2, 0.70f},
-    {"tc 256x192 per CTA pair, 3 stages x 256 B of K", 2, 192, 3, 2, 0.88f},
+    {"tc 128x256 per CTA, 4 stages x 128 B of K", 1, 256, 1, 4, 1, 0.89f},
+    {"tc 128x128 per CTA, 3 stages x 256 B of K", 1, 128, 1, 3, 2, 0.72f},
+    {"tc 256x256 per CTA pair, 3 stages x 256 B of K", 2, 256, 1, 3, 2, 1.00f},
+    {"tc 256x128 per CTA pair, 4 stages x 256 B of K", 2, 128, 1, 4, 2, 0.70f},
+    {"tc 256x192 per CTA pair, 3 stages x 256 B of K", 2, 192, 1, 3, 2, 0.88f},
+    {"tc 256x384 (2 x 192) per CTA pair, 4 stages x 128 B of K", 2, 192, 2, 4, 1, 1.05f},
+    {"tc 256x512 (2 x 256) per CTA pair, 4 stages x 128 B of K", 2, 256, 2, 4, 1, 1.05f},
 };
 constexpr int kNumConfigs = sizeof(kConfigs) / sizeof(kConfigs[0]);
 constexpr int kNoSplitBit = 0x100;        // added to a forced configuration id: no K-split of the partial wave
@@ -516,11 +623,11 @@ constexpr size_t kCounterBytes = 1024;    // per-tile arrival counters at the he
 constexpr int kMaxSplit = 8;              // parts per tile
 constexpr int kMinStagesPerPart = 4;
 
-template <int CG, int BN, int STAGES, int KBS, bool RAW>
+template <int CG, int BNS, int NSUB, int STAGES, int KBS, bool RAW>
 int launch_cfg(const GemmArgs& a, const TcPlan& plan, cudaStream_t st) {
-    using L = SmemLayout<CG, BN, STAGES, KBS>;
-    static_assert(L::DYN_BYTES <= 232448, "shared memory budget");
-    auto kern = gemm_tc_kernel<CG, BN, STAGES, KBS, RAW>;
+    using L = SmemLayout<CG, BNS, NSUB, STAGES, KBS>;
+    static_assert(L::DYN_BYTES <= SMEM_MAX, "shared memory budget");
+    auto kern = gemm_tc_kernel<CG, BNS, NSUB, STAGES, KBS, RAW>;
     static PerDeviceOnce smem_opt_in;
     if (smem_opt_in.run([&] { return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES); }) != cudaSuccess)
         return W8A8_ERR_CUDA;
@@ -552,9 +659,15 @@ int launch_cfg(const GemmArgs& a, const TcPlan& plan, cudaStream_t st) {
     ++na;
     cfg.attrs = attr;
     cfg.numAttrs = na;
+    RunCtl rc{};
+    rc.status = a.status;
+    rc.sticky = sticky_status_word();
+    rc.wait_limit_ns = wait_limit_ns();
+    rc.after_quantizer = a.after_quantizer ? 1 : 0;
+    rc.starve = starve_mode() == kStarveGemm ? 1 : 0;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tm_a, tm_b, tm_out, a.s_tok, a.s_ch, a.bias,
-                                       RAW ? static_cast<int32_t*>(a.out) : nullptr, a.M, a.N, a.K, a.status,
-                                       a.after_quantizer ? 1 : 0, plan.split_tiles, plan.split_parts,
+                                       RAW ? static_cast<int32_t*>(a.out) : nullptr, a.M, a.N, a.K, rc,
+                                       plan.split_tiles, plan.split_parts,
                                        reinterpret_cast<int32_t*>(static_cast<uint8_t*>(a.split_ws) + kCounterBytes),
                                        static_cast<int*>(a.split_ws));
     return e == cudaSuccess ? W8A8_OK : W8A8_ERR_CUDA;
@@ -563,11 +676,13 @@ int launch_cfg(const GemmArgs& a, const TcPlan& plan, cudaStream_t st) {
 template <bool RAW>
 int launch_by_id(const GemmArgs& a, const TcPlan& plan, cudaStream_t st) {
     switch (plan.config) {
-        case 0: return launch_cfg<1, 256, 4, 1, RAW>(a, plan, st);
-        case 1: return launch_cfg<1, 128, 3, 2, RAW>(a, plan, st);
-        case 2: return launch_cfg<2, 256, 3, 2, RAW>(a, plan, st);
-        case 3: return launch_cfg<2, 128, 4, 2, RAW>(a, plan, st);
-        case 4: return launch_cfg<2, 192, 3, 2, RAW>(a, plan, st);
+        case 0: return launch_cfg<1, 256, 1, 4, 1, RAW>(a, plan, st);
+        case 1: return launch_cfg<1, 128, 1, 3, 2, RAW>(a, plan, st);
+        case 2: return launch_cfg<2, 256, 1, 3, 2, RAW>(a, plan, st);
+        case 3: return launch_cfg<2, 128, 1, 4, 2, RAW>(a, plan, st);
+        case 4: return launch_cfg<2, 192, 1, 3, 2, RAW>(a, plan, st);
+        case 5: return launch_cfg<2, 192, 2, 4, 1, RAW>(a, plan, st);
+        case 6: return launch_cfg<2, 256, 2, 4, 1, RAW>(a, plan, st);
         default: return W8A8_ERR_INVALID_ARG;
     }
 }
@@ -583,23 +698,24 @@ TcPlan plan_config(int id, int M, int N, int K, bool allow_split, bool only_if_f
     TcPlan p{};
     p.config = id;
     const int max_groups = sm_count() / c.cg;
-    const long tiles = static_cast<long>((M + BM * c.cg - 1) / (BM * c.cg)) * ((N + c.bn - 1) / c.bn);
+    const int bn = c.bns * c.nsub;
+    const long tiles = static_cast<long>((M + BM * c.cg - 1) / (BM * c.cg)) * ((N + bn - 1) / bn);
     const int whole_waves = static_cast<int>(tiles / max_groups);
     const int rest = static_cast<int>(tiles % max_groups);
     const int kstages = ((K + BK - 1) / BK + c.kbs - 1) / c.kbs;
     int parts = 1;
-    if (allow_split && rest > 0) {
+    if (allow_split && rest > 0 && c.nsub == 1) {      // tiles of two sub-tiles are never cut
         parts = max_groups / rest;
         if (parts > kstages / kMinStagesPerPart) parts = kstages / kMinStagesPerPart;
         if (parts > kMaxSplit) parts = kMaxSplit;
-        const size_t need = kCounterBytes + static_cast<size_t>(rest) * c.cg * c.bn * BM * sizeof(int32_t);
+        const size_t need = kCounterBytes + static_cast<size_t>(rest) * c.cg * bn * BM * sizeof(int32_t);
         if (parts < 2 || need > scratch_bytes) parts = 1;
     }
     // ~20.3 int8 TOPS per SM for configuration 2 in whole waves. A partial wave that is left whole runs its
     // tiles faster than that (measured ~0.72 of the tile time with few SMs active: the operand traffic of a full
     // wave is what holds the rate down); a wave cut along K keeps every SM busy and pays ~10 us for zeroing the
     // slabs, the reductions, the pipeline refill and the read-back.
-    const double tile_us = 2.0 * BM * c.bn * static_cast<double>(K) / 20.3e6 / c.eff;
+    const double tile_us = 2.0 * BM * bn * static_cast<double>(K) / 20.3e6 / c.eff;
     const double fixed_us = 4.0;                       // launch, pipeline fill, last epilogue
     const double whole_rest_us = tile_us * (0.72 + 0.28 * rest / max_groups);
     const double split_rest_us = tile_us / parts + 10.0;
@@ -610,7 +726,7 @@ TcPlan plan_config(int id, int M, int N, int K, bool allow_split, bool only_if_f
         p.split_tiles = rest;
         p.split_parts = parts;
         p.groups = whole_waves > 0 ? max_groups : rest * parts;
-        p.scratch_bytes = kCounterBytes + static_cast<size_t>(rest) * c.cg * c.bn * BM * sizeof(int32_t);
+        p.scratch_bytes = kCounterBytes + static_cast<size_t>(rest) * c.cg * bn * BM * sizeof(int32_t);
     } else {
         p.split_tiles = 0;
         p.split_parts = 0;
@@ -632,10 +748,10 @@ TcPlan tc_plan(int M, int N, int K, int forced, size_t scratch_bytes) {
     const int id = forced < 0 ? -1 : (forced & (kNoSplitBit - 1));
     if (id >= 0 && id < kNumConfigs) return plan_config(id, M, N, K, allow_split, false, scratch_bytes, nullptr);   // forced: cut whenever possible
     // lowest estimated time; on (near) ties the earlier entry of this preference order wins
-    const int order[kNumConfigs] = {2, 0, 4, 3, 1};
+    constexpr int order[] = {2, 0, 4, 3, 1};
     TcPlan best{};
     double best_us = 0.0;
-    for (int i = 0; i < kNumConfigs; ++i) {
+    for (int i = 0; i < static_cast<int>(sizeof(order) / sizeof(order[0])); ++i) {
         double us = 0.0;
         const TcPlan p = plan_config(order[i], M, N, K, allow_split, true, scratch_bytes, &us);
         if (i == 0 || us < best_us * 0.97) { best = p; best_us = us; }

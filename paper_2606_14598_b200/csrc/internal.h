@@ -51,6 +51,18 @@ inline int sm_count() {
 // is a w8a8_status value, the next byte says which wait gave up).
 constexpr int kStatusTimeout = 7;
 
+// ---- api.cu : controls shared by the launchers
+// Bound of every device-side wait in nanoseconds (2 s unless a test lowered it).
+uint64_t wait_limit_ns();
+// Test-only starvation hook: 0 = none; kStarveGemm = the GEMM's producer withholds the first k-stage of its first
+// tile; kStarveQuant = the staged quantizer's producer withholds its first row group. Nothing invalid is touched:
+// the consumers' bounded waits run out, the kernel unwinds and returns, and the status word says which wait gave up.
+constexpr int kStarveGemm = 1, kStarveQuant = 2;
+int starve_mode();
+// Device address, on the current device, of the word that keeps the first time-out of any call until the host
+// reads and clears it (int8_sticky_status); nullptr if it cannot be resolved.
+int* sticky_status_word();
+
 // ---- quantize.cu
 // status_to_clear: workspace status word the kernel resets (or nullptr).
 // mult: per-input-channel factors fp32 [K] multiplied into the operand first (SmoothQuant hook), or nullptr.

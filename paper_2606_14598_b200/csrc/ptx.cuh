@@ -45,7 +45,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // returns false so that the caller can unwind and the CTA can exit cleanly.
 struct WaitCtl {
     volatile int* abort_flag;   // shared memory, one per CTA
-    int* status;                // global status word of the workspace
+    int* status;                // global status word of the workspace (reset by every call)
+    int* sticky;                // device-wide word that keeps the first time-out until the host clears it, or nullptr
     uint64_t limit_ns;
 };
 
@@ -59,6 +60,7 @@ static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity
             if (globaltimer_ns() - t0 > ctl.limit_ns) {
                 *ctl.abort_flag = 1;
                 atomicCAS(ctl.status, 0, status_code | (where << 8));
+                if (ctl.sticky != nullptr) atomicCAS(ctl.sticky, 0, status_code | (where << 8));
                 return false;
             }
         }

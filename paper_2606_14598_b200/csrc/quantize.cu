@@ -158,7 +158,14 @@ constexpr int SG_WARPS = 16;                         // consumer warps per CTA (
 constexpr int SG_THREADS = (SG_WARPS + 1) * 32;
 constexpr int SG_SMEM_BUDGET = 200 * 1024;           // shared memory for the rings of one SM
 constexpr int SG_SMEM_MAX = 226 * 1024;              // all a CTA can have: only for rows too long for the budget above
-constexpr uint64_t SG_WAIT_LIMIT_NS = 2000000000ull; // bounded waits, as everywhere
+
+// Where time-outs go and how long a wait may last (every wait is bounded, as everywhere), plus the test hook.
+struct QuantCtl {
+    int* status;            // workspace status word this kernel resets, or nullptr (standalone quantizer)
+    int* sticky;            // device-wide sticky status word, or nullptr
+    uint64_t wait_limit_ns;
+    int starve;             // test hook: the producer of every CTA withholds its first row group
+};
 
 __device__ __forceinline__ void bulk_load_row(uint32_t smem_dst, const void* gsrc, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -170,8 +177,9 @@ __device__ __forceinline__ void bulk_load_row(uint32_t smem_dst, const void* gsr
 template <int WPR, bool SMOOTH>
 __global__ void __launch_bounds__(SG_THREADS, 2)
 quant_rows_staged_kernel(const __nv_bfloat16* __restrict__ x, int64_t ld, int rows, int K,
-                         int8_t* __restrict__ q, float* __restrict__ s_out, int* status, int num_stages,
+                         int8_t* __restrict__ q, float* __restrict__ s_out, const QuantCtl qc, int num_stages,
                          const float* __restrict__ mult) {
+    int* const status = qc.status;
     // a dependent kernel (the GEMM) may set itself up while this one runs; it waits for this grid before reading
     grid_dep_launch_dependents();
 
@@ -188,7 +196,7 @@ quant_rows_staged_kernel(const __nv_bfloat16* __restrict__ x, int64_t ld, int ro
     float* s_red = reinterpret_cast<float*>(base_ptr + num_stages * stage_bytes + 16 * num_stages);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(s_red + SG_WARPS);
     __shared__ int dummy_status;
-    const WaitCtl ctl{abort_flag, status != nullptr ? status : &dummy_status, SG_WAIT_LIMIT_NS};
+    const WaitCtl ctl{abort_flag, status != nullptr ? status : &dummy_status, qc.sticky, qc.wait_limit_ns};
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
@@ -210,8 +218,15 @@ quant_rows_staged_kernel(const __nv_bfloat16* __restrict__ x, int64_t ld, int ro
         if (lane == 0) {
             int stage = 0;
             uint32_t phase = 0;
+            bool withhold = qc.starve != 0;
             for (int g = blockIdx.x; g < total_groups; g += gridDim.x) {
                 if (!mbar_wait(empty_bar(stage), phase ^ 1u, ctl, 1, kStatusTimeout)) break;
+                if (withhold) {
+                    // test hook: nothing is posted for this stage, so the consumers' bounded wait on it runs out
+                    withhold = false;
+                    if (++stage == num_stages) { stage = 0; phase ^= 1u; }
+                    continue;
+                }
                 const int r0 = g * RPS;
                 const int nr = min(RPS, rows - r0);
                 mbar_arrive_expect_tx(full_bar(stage), nr * row_bytes);
@@ -497,9 +512,10 @@ cudaError_t launch_staged(const __nv_bfloat16* x, int64_t ld, int rows, int K, i
     const int cap = ctas_per_sm * sm_count();
     const int grid = groups < cap ? groups : cap;
     const float* no_mult = nullptr;
+    const QuantCtl qc{status, sticky_status_word(), wait_limit_ns(), starve_mode() == kStarveQuant ? 1 : 0};
     if (mult != nullptr)
-        return launch_pdl(quant_rows_staged_kernel<WPR, true>, grid, SG_THREADS, smem, st, x, ld, rows, K, q, s, status, num_stages, mult);
-    return launch_pdl(quant_rows_staged_kernel<WPR, false>, grid, SG_THREADS, smem, st, x, ld, rows, K, q, s, status, num_stages, no_mult);
+        return launch_pdl(quant_rows_staged_kernel<WPR, true>, grid, SG_THREADS, smem, st, x, ld, rows, K, q, s, qc, num_stages, mult);
+    return launch_pdl(quant_rows_staged_kernel<WPR, false>, grid, SG_THREADS, smem, st, x, ld, rows, K, q, s, qc, num_stages, no_mult);
 }
 
 } // namespace

@@ -18,17 +18,53 @@ def env_world():
             int(os.environ.get("WORLD_SIZE", "1")))
 
 
+RDZV_FILE_ENV = "W8A8_RDZV_FILE"
+
+
 def init(backend: str):
-    """Joins the process group described by RANK / WORLD_SIZE / MASTER_* when there is more than one rank."""
+    """Joins the process group described by RANK / WORLD_SIZE when there is more than one rank. The ranks meet
+    through MASTER_ADDR / MASTER_PORT (a launcher such as torchrun sets them), or, when W8A8_RDZV_FILE names a
+    fresh file, through that file: no port has to be picked ahead of time, so nothing can take it first."""
     rank, local_rank, world = env_world()
     if world > 1 and not dist.is_initialized():
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        os.environ.setdefault("MASTER_PORT", "29500")
         kw = {}
         if backend == "nccl":
             kw["device_id"] = torch.device("cuda", local_rank)
+        rdzv = os.environ.get(RDZV_FILE_ENV)
+        if rdzv:
+            kw["init_method"] = "file://" + rdzv
+        else:
+            os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+            os.environ.setdefault("MASTER_PORT", "29500")
         dist.init_process_group(backend=backend, rank=rank, world_size=world, **kw)
     return rank, local_rank, world
+
+
+def spawn_ranks(argv, world: int, extra_env: dict | None = None, timeout: float | None = None):
+    """Runs `argv` as `world` processes, one per rank (rank i is meant for GPU i), that meet through a rendezvous
+    file. Returns [(returncode, stdout, stderr)] by rank. The children of a failed job are not left behind."""
+    import subprocess
+    import tempfile
+    with tempfile.TemporaryDirectory(prefix="w8a8_rdzv_") as d:
+        procs = []
+        for r in range(world):
+            env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(world))
+            env[RDZV_FILE_ENV] = os.path.join(d, "store")
+            for k in ("MASTER_ADDR", "MASTER_PORT"):
+                env.pop(k, None)
+            env.update(extra_env or {})
+            procs.append(subprocess.Popen(argv, env=env, stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True))
+        out = []
+        try:
+            for p in procs:
+                o, e = p.communicate(timeout=timeout)
+                out.append((p.returncode, o, e))
+        finally:
+            for p in procs:
+                if p.poll() is None:
+                    p.kill()
+                    p.wait()
+        return out
 
 
 def shard_rows(M: int, rank: int, world: int, multiple: int = 1):

@@ -1,7 +1,6 @@
 """World-size-2 CPU (gloo) test of the benchmark's multi-rank plumbing: row sharding covers the tokens
 exactly once, and whole-job throughput is all ranks' units over the slowest rank's time."""
 import os
-import socket
 import subprocess
 import sys
 import textwrap
@@ -32,31 +31,45 @@ WORKER = textwrap.dedent("""
 """) % ROOT
 
 
-def free_port():
-    s = socket.socket()
-    s.bind(("127.0.0.1", 0))
-    p = s.getsockname()[1]
-    s.close()
-    return p
-
-
 def test_two_ranks_gloo():
+    # the ranks meet through a rendezvous file (no port is picked ahead of time, so no other process can take it)
     import json
-    port = str(free_port())
+    from paper_2606_14598_b200.dist import spawn_ranks
+    results = spawn_ranks([sys.executable, "-c", WORKER], 2, extra_env={"OMP_NUM_THREADS": "2"}, timeout=180)
+    outs = []
+    for rc, o, e in results:
+        assert rc == 0, e[-2000:]
+        outs.append(json.loads(o.strip().splitlines()[-1]))
+    outs.sort(key=lambda d: d["rank"])
+    assert outs[0]["lo"] == 0 and outs[0]["hi"] == outs[1]["lo"] and outs[1]["hi"] == 50
+    assert all(d["same"] for d in outs)                      # sharding over tokens changes no bits
+    assert all(d["rows"] == 50.0 and d["tmax"] == 2.0 and d["value"] == 25.0 for d in outs)
+
+
+def test_two_ranks_gloo_through_master_addr_and_port():
+    # the launcher's way (torchrun sets MASTER_ADDR / MASTER_PORT): rank 0 opens the store on a port this test asked
+    # the kernel for while still holding it open with SO_REUSEADDR, which narrows the window in which another process
+    # could take it to the moment between close and bind
+    import json
+    import socket
+    s = socket.socket()
+    s.setsockopt(socket.SOL_SOCKET, socket.SO_REUSEADDR, 1)
+    s.bind(("127.0.0.1", 0))
+    port = str(s.getsockname()[1])
     procs = []
     for r in range(2):
         env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE="2", MASTER_ADDR="127.0.0.1", MASTER_PORT=port,
                    OMP_NUM_THREADS="2")
+        env.pop("W8A8_RDZV_FILE", None)
+        if r == 0:
+            s.close()
         procs.append(subprocess.Popen([sys.executable, "-c", WORKER], env=env, stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True))
     outs = []
     for p in procs:
         o, e = p.communicate(timeout=180)
         assert p.returncode == 0, e[-2000:]
         outs.append(json.loads(o.strip().splitlines()[-1]))
-    outs.sort(key=lambda d: d["rank"])
-    assert outs[0]["lo"] == 0 and outs[0]["hi"] == outs[1]["lo"] and outs[1]["hi"] == 50
-    assert all(d["same"] for d in outs)                      # sharding over tokens changes no bits
-    assert all(d["rows"] == 50.0 and d["tmax"] == 2.0 and d["value"] == 25.0 for d in outs)
+    assert all(d["same"] and d["rows"] == 50.0 for d in outs)
 
 
 def test_shard_rows_partition():
@@ -88,6 +101,15 @@ def test_reference_arm_prints_one_json_line_and_only_on_rank_zero():
     assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] >= 1 and d["cpu_baseline"]["sample"]
     assert d["e2e"]["h2d_bytes_per_step"] == 0 and d["e2e"]["d2h_bytes_per_step"] == 0 and d["gpu_launches"] == 0
     assert d["config"]["workload"].startswith("c1")
-    env1 = dict(env, RANK="1", LOCAL_RANK="1", WORLD_SIZE="2", MASTER_ADDR="127.0.0.1", MASTER_PORT=str(free_port()))
+    env1 = dict(env, RANK="1", LOCAL_RANK="1", WORLD_SIZE="2", MASTER_ADDR="127.0.0.1", MASTER_PORT="29999")
     r1 = subprocess.run(cmd + ["--gpus", "2"], env=env1, capture_output=True, text=True, timeout=300, cwd=ROOT)
     assert r1.returncode == 0 and r1.stdout.strip() == "", r1.stderr[-2000:]
+    # without a launcher `--gpus 2` starts the two ranks itself: still exactly one line, from rank 0
+    r2 = subprocess.run(cmd + ["--gpus", "2"], env=env, capture_output=True, text=True, timeout=300, cwd=ROOT)
+    assert r2.returncode == 0, r2.stderr[-2000:]
+    lines2 = [ln for ln in r2.stdout.splitlines() if ln.strip()]
+    assert len(lines2) == 1 and json.loads(lines2[0])["n_gpus"] == 2 and json.loads(lines2[0])["impl"] == "reference"
+    # the reference arm times exactly --steps steps after --warmup untimed ones
+    r3 = subprocess.run(cmd[:-4] + ["--steps", "4", "--warmup", "2"], env=env, capture_output=True, text=True, timeout=300, cwd=ROOT)
+    d3 = json.loads(r3.stdout.strip().splitlines()[-1])
+    assert d3["steps"] == 4 and d3["warmup"] == 2
