@@ -55,6 +55,10 @@ def _load():
         lib.oracle_quantize_weight_per_channel_smooth.restype = None
         lib.oracle_quantize_act_per_token_smooth.argtypes = [vp, i64, i64, i64, vp, vp, vp]
         lib.oracle_quantize_act_per_token_smooth.restype = None
+        lib.oracle_row_absmax_bf16.argtypes = [vp, i64, i64, i64, vp]
+        lib.oracle_row_absmax_bf16.restype = None
+        lib.oracle_quantize_act_per_token_given_absmax.argtypes = [vp, i64, i64, i64, vp, vp, vp]
+        lib.oracle_quantize_act_per_token_given_absmax.restype = None
         lib.oracle_gemm_i32.argtypes = [vp, vp, vp, i64, i64, i64]
         lib.oracle_gemm_i32.restype = i64
         lib.oracle_epilogue.argtypes = [vp, vp, vp, vp, vp, i64, i64]
@@ -114,6 +118,27 @@ def quantize_act_per_token(A_bits: np.ndarray):
     qa = np.empty((M, K), np.int8)
     s_tok = np.empty((M,), np.float32)
     _load().oracle_quantize_act_per_token(_p(A_bits), M, K, lda, _p(qa), _p(s_tok))
+    return qa, s_tok
+
+
+def row_absmax_bf16(X_bits: np.ndarray) -> np.ndarray:
+    """bf16 bit patterns uint16 [M,N] (rows may be strided) -> fp32 [M], the largest magnitude of every row."""
+    X_bits, ld = _chk_rows(X_bits, np.uint16)
+    M, N = X_bits.shape
+    rowmax = np.empty((M,), np.float32)
+    _load().oracle_row_absmax_bf16(_p(X_bits), M, N, ld, _p(rowmax))
+    return rowmax
+
+
+def quantize_act_per_token_given_absmax(A_bits: np.ndarray, rowmax: np.ndarray):
+    """The quantizer's second half: bf16 bit patterns [M,K] and the absmax of every row fp32 [M] -> (int8 [M,K], fp32 [M])."""
+    A_bits, lda = _chk_rows(A_bits, np.uint16)
+    rowmax = _chk(rowmax, np.float32, 1)
+    M, K = A_bits.shape
+    assert rowmax.shape == (M,)
+    qa = np.empty((M, K), np.int8)
+    s_tok = np.empty((M,), np.float32)
+    _load().oracle_quantize_act_per_token_given_absmax(_p(A_bits), M, K, lda, _p(rowmax), _p(qa), _p(s_tok))
     return qa, s_tok
 
 

@@ -70,19 +70,31 @@ inline int32_t rne_to_int(float v) {
 
 inline int32_t clamp127(int32_t q) { return q > 127 ? 127 : (q < -127 ? -127 : q); }
 
-// One row of the symmetric absmax quantizer on fp32 values.
-void quant_row(const float* x, int64_t K, int8_t* q, float* s_out) {
+// max_k |x[k]| of one row (exact; 0 for an empty or all-zero row).
+float row_absmax(const float* x, int64_t K) {
     float amax = 0.0f;
     for (int64_t k = 0; k < K; ++k) {
         float a = std::fabs(x[k]);
         if (a > amax) amax = a;
     }
+    return amax;
+}
+
+// The second half of the quantizer: scale and codes of one row from an absmax that is handed in. With the row's
+// own absmax this is the whole quantizer; with a larger one the codes use less of the range; with a smaller one the
+// clamp binds.
+void quant_row_given(const float* x, int64_t K, float amax, int8_t* q, float* s_out) {
     float s = (amax > 0.0f) ? amax / 127.0f : 1.0f;
     for (int64_t k = 0; k < K; ++k) {
         float r = x[k] / s;
         q[k] = int8_t(clamp127(rne_to_int(r)));
     }
     *s_out = s;
+}
+
+// One row of the symmetric absmax quantizer on fp32 values.
+void quant_row(const float* x, int64_t K, int8_t* q, float* s_out) {
+    quant_row_given(x, K, row_absmax(x, K), q, s_out);
 }
 
 } // namespace
@@ -136,6 +148,35 @@ void oracle_quantize_act_per_token(const uint16_t* A, int64_t M, int64_t K, int6
         float* row = new float[K > 0 ? K : 1];
         for (int64_t k = 0; k < K; ++k) row[k] = bf16_to_f32(A[m * lda + k]);
         quant_row(row, K, qa + m * K, s_tok + m);
+        delete[] row;
+    }
+}
+
+// The quantizer fused into its producer (the paper's Method: per-token scales are dynamic, computed online from the
+// activations; nothing says in how many passes). Two pieces:
+//   * the producer of an activation matrix also reports, per token, the largest magnitude it wrote:
+//     rowmax[m] = max_n |X[m,n]| over the bf16 values as stored (exact, order-free);
+//   * the quantizer takes that number instead of searching for it (one pass over the row).
+// With rowmax equal to the row's absmax the result is, by construction, that of oracle_quantize_act_per_token.
+void oracle_row_absmax_bf16(const uint16_t* X, int64_t M, int64_t N, int64_t ld, float* rowmax) {
+    #pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m) {
+        float amax = 0.0f;
+        for (int64_t n = 0; n < N; ++n) {
+            float a = std::fabs(bf16_to_f32(X[m * ld + n]));
+            if (a > amax) amax = a;
+        }
+        rowmax[m] = amax;
+    }
+}
+
+void oracle_quantize_act_per_token_given_absmax(const uint16_t* A, int64_t M, int64_t K, int64_t lda, const float* rowmax,
+                                                int8_t* qa, float* s_tok) {
+    #pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m) {
+        float* row = new float[K > 0 ? K : 1];
+        for (int64_t k = 0; k < K; ++k) row[k] = bf16_to_f32(A[m * lda + k]);
+        quant_row_given(row, K, rowmax[m], qa + m * K, s_tok + m);
         delete[] row;
     }
 }

@@ -157,6 +157,40 @@ def test_quantizer_leading_dimension_is_honoured():
     assert (ss == (np.abs(bits_to_f64(np.ascontiguousarray(sl))).max(axis=1) / 127.0).astype(np.float32)).all()
 
 
+def test_row_absmax_and_quantizer_with_the_absmax_handed_in():
+    # row absmax: hand vectors (the largest magnitude is negative; a minus zero; an all-zero row), then numpy
+    x = np.array([[1, -3, 2, -0.0], [0, 0, 0, 0], [0.5, 0.25, -0.125, 0.5]], np.float32)
+    assert oracle.row_absmax_bf16(bf16_bits_of(x)).tolist() == [3.0, 0.0, 0.5]
+    rng = np.random.default_rng(23)
+    a = rng.standard_normal((40, 300)).astype(np.float32)
+    a[:, 5] *= 20
+    a[7] = 0
+    bits = bf16_bits_of(a)
+    assert (oracle.row_absmax_bf16(bits) == np.abs(bits_to_f64(bits)).max(axis=1).astype(np.float32)).all()
+    wide = np.zeros((40, 330), np.uint16)
+    wide[:, :] = bf16_bits_of(np.full((40, 330), 1000.0, np.float32))
+    wide[:, 10:310] = bits
+    assert (oracle.row_absmax_bf16(wide[:, 10:310]) == oracle.row_absmax_bf16(bits)).all()     # row stride honoured
+    # handed the row's own absmax, the one-pass quantizer is the two-pass quantizer, on every row (zero row included)
+    q2, s2 = oracle.quantize_act_per_token(bits)
+    q1, s1 = oracle.quantize_act_per_token_given_absmax(bits, oracle.row_absmax_bf16(bits))
+    assert (q1 == q2).all() and (s1.view(np.uint32) == s2.view(np.uint32)).all() and s1[7] == 1.0
+    # hand vectors: absmax 127 handed in => s = 1 and q = rne(x), ties to even
+    t = np.array([[100, 0.5, 1.5, 2.5, -0.5, -1.5, -2.5, 63.5]], np.float32)
+    q, s = oracle.quantize_act_per_token_given_absmax(bf16_bits_of(t), np.array([127.0], np.float32))
+    assert s[0] == 1.0 and q.tolist() == [[100, 0, 2, 2, 0, -2, -2, 64]]
+    # a larger absmax than the row has: s = 2, q = rne(x / 2); the range is only half used
+    u = np.array([[127, 1, 3, 5, -7, 126, 0, -127]], np.float32)
+    q, s = oracle.quantize_act_per_token_given_absmax(bf16_bits_of(u), np.array([254.0], np.float32))
+    assert s[0] == 2.0 and q.tolist() == [[64, 0, 2, 2, -4, 63, 0, -64]]
+    # a smaller one: the clamp binds at +-127 (and -128 is never produced)
+    q, s = oracle.quantize_act_per_token_given_absmax(bf16_bits_of(u), np.array([63.5], np.float32))
+    assert s[0] == 0.5 and q.tolist() == [[127, 2, 6, 10, -14, 127, 0, -127]]
+    # zero handed in: s = 1
+    q, s = oracle.quantize_act_per_token_given_absmax(bf16_bits_of(u), np.array([0.0], np.float32))
+    assert s[0] == 1.0 and q.tolist() == [[127, 1, 3, 5, -7, 126, 0, -127]]
+
+
 # --------------------------------------------------------------------------- integer GEMM
 
 def brute_gemm(qa, qw):
