@@ -445,6 +445,11 @@ def main():
             g_args = [fused_args(L, bf16=False, s_tok=st_, qa=qa_, ws=ws8) for (L, st_, qa_) in views]
             q_args = [(L["A"].data_ptr(), M, K, K, qa_.data_ptr(), st_.data_ptr(), stream) for (L, st_, qa_) in views]
             f_args = [fused_args(L) for (L, _, _) in views]
+            # the one-pass quantizer takes the absmax of every row from the producer of the activations; here the set-up
+            # computes it (exactly: bf16 widens to fp32 without rounding and a maximum does not round)
+            rowmax = [L["A"].float().abs().amax(dim=1).contiguous() for (L, _, _) in views]
+            q1_args = [(L["A"].data_ptr(), M, K, K, rm.data_ptr(), qa_.data_ptr(), st_.data_ptr(), stream)
+                       for (L, st_, qa_), rm in zip(views, rowmax)]
 
             def gemm_only():
                 it[0] += 1
@@ -456,6 +461,10 @@ def main():
             def quant_only():
                 it[0] += 1
                 raw.int8_quantize_act_per_token(*q_args[it[0] % len(q_args)])
+
+            def quant_one_pass():
+                it[0] += 1
+                raw.int8_quantize_act_per_token_given_absmax(*q1_args[it[0] % len(q1_args)])
 
             def fused():
                 it[0] += 1
@@ -478,6 +487,7 @@ def main():
             stamp = w8.gemm_clock_stamps(ws8) if M > 8 else None
             tgh = batch_time(gemm_hot)
             tq = batch_time(quant_only)
+            tq1 = batch_time(quant_one_pass)
             tf_ = batch_time(fused)
             plan = w8.int8_linear_plan(M, N, K, w8.ACT_BF16, rot[0]["ws"].numel())
             per_shape.append({"name": spec.name, "M": M, "K": K, "N": N,
@@ -489,7 +499,9 @@ def main():
                               "gemm_sm_mhz": stamp[0] if stamp else None,
                               "gemm_first_cta_us": stamp[1] * 1e6 if stamp else None,
                               "gemm_epilogue_hot_l2_us": tgh * 1e6, "gemm_epilogue_hot_l2_tops": spec.ops / tgh / 1e12,
-                              "quantizer_us": tq * 1e6, "quantizer_gbs": model.quantizer_bytes(M, K) / tq / 1e9})
+                              "quantizer_us": tq * 1e6, "quantizer_gbs": model.quantizer_bytes(M, K) / tq / 1e9,
+                              "quantizer_given_absmax_us": tq1 * 1e6,
+                              "quantizer_given_absmax_gbs": (model.quantizer_bytes(M, K) + 4 * M) / tq1 / 1e9})
             if M > 16:
                 gemm_ops += spec.ops
                 gemm_sec += tg

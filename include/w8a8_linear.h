@@ -148,6 +148,39 @@ int int8_linear_fused_smooth(const void* A_bf16, int64_t lda, const float* a_mul
                              void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The activation quantizer fused into the producer of the activations, as far as it can be stated exactly
+ * (Method, "The fused kernel": the per-token scales are dynamic, computed online from the activations; the paper
+ * does not say in how many passes). The quantizer's first pass only finds the largest magnitude of every token.
+ * A producer that writes the activations can report that number on the way, and the quantizer then needs one pass:
+ *
+ * int8_linear_fused_rowmax
+ *     int8_linear_fused that additionally writes rowmax_out[m] = max_n |out[m,n]|, the largest magnitude among the
+ *     bf16 values it stored for token m (fp32 [M], device; exact: the maximum does not depend on the order).
+ *     rowmax_out is zeroed by a memset on `stream` ahead of the kernels and merged with atomic maxima.
+ * int8_quantize_act_per_token_given_absmax
+ *     int8_quantize_act_per_token with the absmax of every row handed in: s = rowmax[m] > 0 ? rowmax[m] / 127 : 1,
+ *     q = rne(x / s). PRECONDITION: rowmax[m] >= max_k |A[m,k]| and finite. Handed the row's own absmax the results
+ *     equal int8_quantize_act_per_token's bit for bit; a larger value uses less of the int8 range; with a smaller
+ *     one the codes of the elements above it are unspecified (the search pass is what would have caught them).
+ * int8_linear_fused_given_absmax
+ *     int8_linear_fused on bf16 activations whose quantizer takes rowmax_in [M] as above; rowmax_out may be NULL or,
+ *     to chain linears, a buffer that does not overlap rowmax_in (W8A8_ERR_INVALID_ARG otherwise).
+ * A chain y = L2(L1(x)) then runs L1 with _rowmax and L2 with _given_absmax on the same vector. An activation
+ * function between the two (the MLP's GELU) stays with the caller: the kernel that applies it reports the row
+ * maxima of what it writes. All other arguments, requirements and errors as for the plain entry points.
+ */
+int int8_linear_fused_rowmax(const void* A, int a_dtype, int64_t lda, const float* s_tok_in,
+                             const int8_t* qw, const float* s_ch, const float* bias,
+                             void* out_bf16, int64_t ldo, float* rowmax_out, int64_t M, int64_t N, int64_t K,
+                             void* workspace, size_t workspace_bytes, void* stream);
+int int8_quantize_act_per_token_given_absmax(const void* A_bf16, int64_t M, int64_t K, int64_t lda, const float* rowmax,
+                                             int8_t* qa, float* s_tok, void* stream);
+int int8_linear_fused_given_absmax(const void* A_bf16, int64_t lda, const float* rowmax_in,
+                                   const int8_t* qw, const float* s_ch, const float* bias,
+                                   void* out_bf16, int64_t ldo, float* rowmax_out, int64_t M, int64_t N, int64_t K,
+                                   void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Same computation with the activations and the result in HOST memory
  * (pinned memory makes the copies asynchronous): copies A to d_A, runs
  * int8_linear_fused on bf16 activations, copies the result to out_host, all on
@@ -254,7 +287,9 @@ int int8_debug_set_starve(int mode);
 /*
  * Force a kernel configuration for sweeps and tests. -1 = choose from the shape; -2 = choose from the shape
  * but never cut tiles along K; id = that configuration; id + 0x100 = that configuration, never cut along K.
- * Returns the previous value.
+ * For the configuration whose tiles are two sub-tiles side by side, bits 12-19, if not zero, are 1 + the number of
+ * such wide tiles per block of 256 rows (the remaining column blocks run as single sub-tiles); too large a
+ * number falls back to the library's choice. Returns the previous value.
  */
 int int8_linear_force_config(int config_id);
 

@@ -28,6 +28,7 @@ EXPORTS = (
     "int8_status_string", "int8_linear_fused_static", "int8_quantize_weight_per_channel_smooth",
     "int8_quantize_act_per_token_smooth", "int8_linear_fused_smooth", "int8_linear_workspace_min_bytes", "int8_linear_plan",
     "int8_sticky_status", "int8_debug_set_wait_limit_ns", "int8_debug_set_starve",
+    "int8_linear_fused_rowmax", "int8_quantize_act_per_token_given_absmax", "int8_linear_fused_given_absmax",
 )
 
 if not os.path.exists(LIB_PATH):
@@ -62,6 +63,12 @@ _lib.int8_quantize_act_per_token_smooth.argtypes = [_vp, _i64, _i64, _i64, _vp, 
 _lib.int8_quantize_act_per_token_smooth.restype = _int
 _lib.int8_linear_fused_smooth.argtypes = [_vp, _i64, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i64, _vp, _sz, _vp]
 _lib.int8_linear_fused_smooth.restype = _int
+_lib.int8_linear_fused_rowmax.argtypes = [_vp, _int, _i64, _vp, _vp, _vp, _vp, _vp, _i64, _vp, _i64, _i64, _i64, _vp, _sz, _vp]
+_lib.int8_linear_fused_rowmax.restype = _int
+_lib.int8_quantize_act_per_token_given_absmax.argtypes = [_vp, _i64, _i64, _i64, _vp, _vp, _vp, _vp]
+_lib.int8_quantize_act_per_token_given_absmax.restype = _int
+_lib.int8_linear_fused_given_absmax.argtypes = [_vp, _i64, _vp, _vp, _vp, _vp, _vp, _i64, _vp, _i64, _i64, _i64, _vp, _sz, _vp]
+_lib.int8_linear_fused_given_absmax.restype = _int
 _lib.int8_gemm_i32_debug.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64, _vp, _sz, _vp]
 _lib.int8_gemm_i32_debug.restype = _int
 _lib.int8_check_status.argtypes = [_vp, _vp]
@@ -207,6 +214,54 @@ def int8_linear_fused_smooth(A: torch.Tensor, a_mult: torch.Tensor, qw: torch.Te
                                          out.stride(0), M, N, K, _ptr(workspace), workspace.numel(), _stream(A)),
            "int8_linear_fused_smooth")
     return out
+
+
+def int8_quantize_act_per_token_given_absmax(A: torch.Tensor, rowmax: torch.Tensor):
+    """One-pass quantizer: bf16 [M,K] and the absmax of every row fp32 [M] (>= the true one) -> (int8 [M,K], fp32 [M])."""
+    _need(A, torch.bfloat16, "A", 2)
+    _need(rowmax, torch.float32, "rowmax", 1)
+    M, K = A.shape
+    if rowmax.shape[0] != M:
+        raise ValueError("rowmax must have M entries")
+    qa = torch.empty((M, K), dtype=torch.int8, device=A.device)
+    s_tok = torch.empty((M,), dtype=torch.float32, device=A.device)
+    _check(_lib.int8_quantize_act_per_token_given_absmax(_ptr(A), M, K, A.stride(0), _ptr(rowmax), _ptr(qa), _ptr(s_tok),
+                                                         _stream(A)), "int8_quantize_act_per_token_given_absmax")
+    return qa, s_tok
+
+
+def int8_linear_fused_rowmax(A: torch.Tensor, qw: torch.Tensor, s_ch: torch.Tensor, bias: torch.Tensor | None = None,
+                             s_tok: torch.Tensor | None = None, out: torch.Tensor | None = None,
+                             workspace: torch.Tensor | None = None, rowmax_in: torch.Tensor | None = None):
+    """Fused linear that also returns rowmax[m] = max_n |out[m,n]| (fp32 [M]). With rowmax_in (bf16 activations only)
+    the quantizer runs in one pass on the absmax handed in. Returns (out, rowmax)."""
+    a_dtype = ACT_BF16 if A.dtype == torch.bfloat16 else ACT_INT8
+    _need(A, torch.bfloat16 if a_dtype == ACT_BF16 else torch.int8, "A", 2)
+    _need(qw, torch.int8, "qw", 2)
+    _need(s_ch, torch.float32, "s_ch", 1)
+    M, K = A.shape
+    N = qw.shape[0]
+    if qw.shape[1] != K or s_ch.shape[0] != N or not qw.is_contiguous():
+        raise ValueError("shape mismatch")
+    if bias is not None:
+        _need(bias, torch.float32, "bias", 1)
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=A.device)
+    if workspace is None:
+        workspace = alloc_workspace(M, N, K, a_dtype, A.device)
+    rowmax = torch.empty((M,), dtype=torch.float32, device=A.device)
+    if rowmax_in is None:
+        _check(_lib.int8_linear_fused_rowmax(_ptr(A), a_dtype, A.stride(0), _ptr(s_tok), _ptr(qw), _ptr(s_ch), _ptr(bias),
+                                             _ptr(out), out.stride(0), _ptr(rowmax), M, N, K, _ptr(workspace),
+                                             workspace.numel(), _stream(A)), "int8_linear_fused_rowmax")
+    else:
+        _need(rowmax_in, torch.float32, "rowmax_in", 1)
+        if a_dtype != ACT_BF16 or rowmax_in.shape[0] != M:
+            raise ValueError("rowmax_in goes with bf16 activations and has M entries")
+        _check(_lib.int8_linear_fused_given_absmax(_ptr(A), A.stride(0), _ptr(rowmax_in), _ptr(qw), _ptr(s_ch), _ptr(bias),
+                                                   _ptr(out), out.stride(0), _ptr(rowmax), M, N, K, _ptr(workspace),
+                                                   workspace.numel(), _stream(A)), "int8_linear_fused_given_absmax")
+    return out, rowmax
 
 
 def int8_linear_workspace_bytes(M: int, N: int, K: int, a_dtype: int = ACT_BF16) -> int:

@@ -137,13 +137,13 @@ static int quantize_weight_impl(const float* W, int64_t N, int64_t K, int64_t ld
     return ce == cudaSuccess ? W8A8_OK : W8A8_ERR_CUDA;
 }
 
-static int quantize_act_impl(const void* A_bf16, int64_t M, int64_t K, int64_t lda, const float* mult,
+static int quantize_act_impl(const void* A_bf16, int64_t M, int64_t K, int64_t lda, const float* mult, const float* amax,
                              int8_t* qa, float* s_tok, void* stream) {
     if (A_bf16 == nullptr || qa == nullptr || s_tok == nullptr) return W8A8_ERR_INVALID_ARG;
     if (M <= 0 || K <= 0 || M > INT32_MAX || K > INT32_MAX || lda < K) return W8A8_ERR_INVALID_ARG;
     if (K % 16 != 0 || lda % 8 != 0 || !aligned16(A_bf16) || !aligned16(qa) || !aligned16(mult)) return W8A8_ERR_ALIGNMENT;
     if (int e = check_arch()) return e;
-    cudaError_t ce = launch_quantize_bf16(A_bf16, lda, static_cast<int>(M), static_cast<int>(K), mult, qa, s_tok, nullptr,
+    cudaError_t ce = launch_quantize_bf16(A_bf16, lda, static_cast<int>(M), static_cast<int>(K), mult, amax, qa, s_tok, nullptr,
                                           static_cast<cudaStream_t>(stream));
     return ce == cudaSuccess ? W8A8_OK : W8A8_ERR_CUDA;
 }
@@ -161,13 +161,19 @@ int int8_quantize_weight_per_channel_smooth(const float* W, int64_t N, int64_t K
 
 int int8_quantize_act_per_token(const void* A_bf16, int64_t M, int64_t K, int64_t lda,
                                 int8_t* qa, float* s_tok, void* stream) {
-    return quantize_act_impl(A_bf16, M, K, lda, nullptr, qa, s_tok, stream);
+    return quantize_act_impl(A_bf16, M, K, lda, nullptr, nullptr, qa, s_tok, stream);
+}
+
+int int8_quantize_act_per_token_given_absmax(const void* A_bf16, int64_t M, int64_t K, int64_t lda, const float* rowmax,
+                                             int8_t* qa, float* s_tok, void* stream) {
+    if (rowmax == nullptr) return W8A8_ERR_INVALID_ARG;
+    return quantize_act_impl(A_bf16, M, K, lda, nullptr, rowmax, qa, s_tok, stream);
 }
 
 int int8_quantize_act_per_token_smooth(const void* A_bf16, int64_t M, int64_t K, int64_t lda, const float* a_mult,
                                        int8_t* qa, float* s_tok, void* stream) {
     if (a_mult == nullptr) return W8A8_ERR_INVALID_ARG;
-    return quantize_act_impl(A_bf16, M, K, lda, a_mult, qa, s_tok, stream);
+    return quantize_act_impl(A_bf16, M, K, lda, a_mult, nullptr, qa, s_tok, stream);
 }
 
 size_t int8_linear_workspace_min_bytes(int64_t M, int64_t N, int64_t K, int a_dtype) {
@@ -215,9 +221,11 @@ void int8_linear_workspace_offsets(int64_t M, int64_t K, size_t* s_tok_offset, s
     if (qa_offset) *qa_offset = q_off;
 }
 
-static int fused_impl(const void* A, int a_dtype, int64_t lda, const float* s_tok_in, const float* a_mult,
+// a_mult: SmoothQuant factors for bf16 activations, or nullptr. amax_in: the absmax of every row of bf16 activations,
+// handed in (one-pass quantizer), or nullptr. rowmax_out: receives the absmax of every output row, or nullptr.
+static int fused_impl(const void* A, int a_dtype, int64_t lda, const float* s_tok_in, const float* a_mult, const float* amax_in,
                       const int8_t* qw, const float* s_ch, const float* bias,
-                      void* out_bf16, int64_t ldo, int64_t M, int64_t N, int64_t K,
+                      void* out_bf16, int64_t ldo, float* rowmax_out, int64_t M, int64_t N, int64_t K,
                       void* workspace, size_t workspace_bytes, void* stream) {
     if (A == nullptr || qw == nullptr || s_ch == nullptr || out_bf16 == nullptr) return W8A8_ERR_INVALID_ARG;
     if (!aligned16(a_mult)) return W8A8_ERR_ALIGNMENT;
@@ -247,8 +255,12 @@ static int fused_impl(const void* A, int a_dtype, int64_t lda, const float* s_to
         if (plan.split_parts >= 2 && cudaMemsetAsync(ws + scratch_off, 0, plan.scratch_bytes, st) != cudaSuccess)
             return W8A8_ERR_CUDA;
     }
+    // the row maxima are merged with atomic maxima by every tile of a row block: they start at zero
+    if (rowmax_out != nullptr && cudaMemsetAsync(rowmax_out, 0, static_cast<size_t>(M) * sizeof(float), st) != cudaSuccess)
+        return W8A8_ERR_CUDA;
 
     GemmArgs g{};
+    g.rowmax = rowmax_out;
     g.qw = qw; g.s_ch = s_ch; g.bias = bias; g.out = out_bf16; g.ldo = ldo;
     g.M = static_cast<int>(M); g.N = static_cast<int>(N); g.K = static_cast<int>(K);
     g.raw_i32 = false; g.status = status; g.split_ws = plan.split_parts >= 2 ? ws + scratch_off : nullptr;
@@ -259,7 +271,7 @@ static int fused_impl(const void* A, int a_dtype, int64_t lda, const float* s_to
         int8_t* qa = reinterpret_cast<int8_t*>(ws + q_off);
         // the quantizer clears the status word; the GEMM behind it (programmatic dependent launch) sets
         // itself up while the quantizer runs and waits for it before its first read
-        if (launch_quantize_bf16(A, lda, g.M, g.K, a_mult, qa, s_tok, status, st) != cudaSuccess) return W8A8_ERR_CUDA;
+        if (launch_quantize_bf16(A, lda, g.M, g.K, a_mult, amax_in, qa, s_tok, status, st) != cudaSuccess) return W8A8_ERR_CUDA;
         g.qa = qa; g.lda_q = K; g.s_tok = s_tok; g.after_quantizer = true;
     } else {
         g.qa = static_cast<const int8_t*>(A); g.lda_q = lda; g.s_tok = s_tok_in; g.after_quantizer = false;
@@ -272,7 +284,31 @@ int int8_linear_fused(const void* A, int a_dtype, int64_t lda, const float* s_to
                       const int8_t* qw, const float* s_ch, const float* bias,
                       void* out_bf16, int64_t ldo, int64_t M, int64_t N, int64_t K,
                       void* workspace, size_t workspace_bytes, void* stream) {
-    return fused_impl(A, a_dtype, lda, s_tok_in, nullptr, qw, s_ch, bias, out_bf16, ldo, M, N, K,
+    return fused_impl(A, a_dtype, lda, s_tok_in, nullptr, nullptr, qw, s_ch, bias, out_bf16, ldo, nullptr, M, N, K,
+                      workspace, workspace_bytes, stream);
+}
+
+int int8_linear_fused_rowmax(const void* A, int a_dtype, int64_t lda, const float* s_tok_in,
+                             const int8_t* qw, const float* s_ch, const float* bias,
+                             void* out_bf16, int64_t ldo, float* rowmax_out, int64_t M, int64_t N, int64_t K,
+                             void* workspace, size_t workspace_bytes, void* stream) {
+    if (rowmax_out == nullptr) return W8A8_ERR_INVALID_ARG;
+    return fused_impl(A, a_dtype, lda, s_tok_in, nullptr, nullptr, qw, s_ch, bias, out_bf16, ldo, rowmax_out, M, N, K,
+                      workspace, workspace_bytes, stream);
+}
+
+int int8_linear_fused_given_absmax(const void* A_bf16, int64_t lda, const float* rowmax_in,
+                                   const int8_t* qw, const float* s_ch, const float* bias,
+                                   void* out_bf16, int64_t ldo, float* rowmax_out, int64_t M, int64_t N, int64_t K,
+                                   void* workspace, size_t workspace_bytes, void* stream) {
+    if (rowmax_in == nullptr) return W8A8_ERR_INVALID_ARG;
+    if (rowmax_out != nullptr && M > 0) {
+        // the output maxima are zeroed before the quantizer reads the input maxima: the two must not share memory
+        const uintptr_t a = reinterpret_cast<uintptr_t>(rowmax_in), b = reinterpret_cast<uintptr_t>(rowmax_out);
+        const uintptr_t bytes = static_cast<uintptr_t>(M) * sizeof(float);
+        if (a < b + bytes && b < a + bytes) return W8A8_ERR_INVALID_ARG;
+    }
+    return fused_impl(A_bf16, W8A8_ACT_BF16, lda, nullptr, nullptr, rowmax_in, qw, s_ch, bias, out_bf16, ldo, rowmax_out, M, N, K,
                       workspace, workspace_bytes, stream);
 }
 
@@ -281,7 +317,7 @@ int int8_linear_fused_smooth(const void* A_bf16, int64_t lda, const float* a_mul
                              void* out_bf16, int64_t ldo, int64_t M, int64_t N, int64_t K,
                              void* workspace, size_t workspace_bytes, void* stream) {
     if (a_mult == nullptr) return W8A8_ERR_INVALID_ARG;
-    return fused_impl(A_bf16, W8A8_ACT_BF16, lda, nullptr, a_mult, qw, s_ch, bias, out_bf16, ldo, M, N, K,
+    return fused_impl(A_bf16, W8A8_ACT_BF16, lda, nullptr, a_mult, nullptr, qw, s_ch, bias, out_bf16, ldo, nullptr, M, N, K,
                       workspace, workspace_bytes, stream);
 }
 

@@ -23,9 +23,10 @@ __device__ __forceinline__ int dot16(const uint4& a, const uint4& b, int acc) {
 
 template <int MB, int NPW, int WARPS>
 __global__ void __launch_bounds__(WARPS * 32)
-gemm_simt_kernel(const int8_t* __restrict__ qa, int64_t lda_q, const float* __restrict__ s_tok,
+gemm_simt_kernel(const int8_t* qa, int64_t lda_q, const float* s_tok,
                  const int8_t* __restrict__ qw, const float* __restrict__ s_ch, const float* __restrict__ bias,
-                 void* __restrict__ out, int64_t ldo, int M, int N, int K, int raw_i32, int after_quantizer, int* status) {
+                 void* __restrict__ out, int64_t ldo, int M, int N, int K, int raw_i32, int after_quantizer, int* status,
+                 float* rowmax) {
     grid_dep_launch_dependents();      // a following kernel launched to allow it may set itself up early
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n0 = (blockIdx.x * WARPS + warp) * NPW;
@@ -56,7 +57,7 @@ gemm_simt_kernel(const int8_t* __restrict__ qa, int64_t lda_q, const float* __re
 #pragma unroll
         for (int j = 0; j < NPW; ++j) w[j] = __ldg(reinterpret_cast<const uint4*>(wrow[j] + k));
 #pragma unroll
-        for (int i = 0; i < MB; ++i) a[i] = *reinterpret_cast<const uint4*>(arow[i] + k);
+        for (int i = 0; i < MB; ++i) a[i] = __ldcg(reinterpret_cast<const uint4*>(arow[i] + k));
 #pragma unroll
         for (int i = 0; i < MB; ++i)
 #pragma unroll
@@ -83,10 +84,15 @@ gemm_simt_kernel(const int8_t* __restrict__ qa, int64_t lda_q, const float* __re
                 static_cast<int32_t*>(out)[static_cast<int64_t>(m) * ldo + n] = mine;
             } else {
                 float t = __int2float_rn(mine);
-                t = __fmul_rn(t, s_tok[m]);
+                t = __fmul_rn(t, __ldcg(s_tok + m));      // plain loads for what the quantizer ahead of this kernel wrote
                 t = __fmul_rn(t, s_ch[n]);
                 if (bias != nullptr) t = __fadd_rn(t, bias[n]);
-                static_cast<__nv_bfloat16*>(out)[static_cast<int64_t>(m) * ldo + n] = __float2bfloat16_rn(t);
+                const __nv_bfloat16 o = __float2bfloat16_rn(t);
+                static_cast<__nv_bfloat16*>(out)[static_cast<int64_t>(m) * ldo + n] = o;
+                if (rowmax != nullptr) {      // side output: largest magnitude written to row m (non-negative floats order like their bits)
+                    const uint32_t bits = (static_cast<uint32_t>(*reinterpret_cast<const uint16_t*>(&o)) & 0x7fffu) << 16;
+                    if (bits != 0u) atomicMax(reinterpret_cast<unsigned int*>(rowmax) + m, bits);
+                }
             }
         }
     }
@@ -106,7 +112,8 @@ cudaError_t launch(const GemmArgs& a, cudaStream_t st) {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, gemm_simt_kernel<MB, NPW, WARPS>, a.qa, a.lda_q, a.s_tok, a.qw, a.s_ch, a.bias,
-                              a.out, a.ldo, a.M, a.N, a.K, a.raw_i32 ? 1 : 0, a.after_quantizer ? 1 : 0, a.status);
+                              a.out, a.ldo, a.M, a.N, a.K, a.raw_i32 ? 1 : 0, a.after_quantizer ? 1 : 0, a.status,
+                              a.raw_i32 ? static_cast<float*>(nullptr) : a.rowmax);
 }
 
 } // namespace

@@ -118,7 +118,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                const __grid_constant__ CUtensorMap tm_out,
                const float* s_tok, const float* __restrict__ s_ch, const float* __restrict__ bias,
                int32_t* __restrict__ raw_out, int M, int N, int K, const RunCtl rc,
-               int split_tiles, int split_s, int32_t* split_slabs, int* split_counters) {
+               int split_tiles, int split_s, int32_t* split_slabs, int* split_counters, int wide_per_row,
+               float* rowmax) {
     using L = SmemLayout<CG, BNS, NSUB, STAGES, KBS>;
     constexpr int BN = L::BN;
     // the next kernel in the stream, if it was launched to allow it (the next call's quantizer is), may be scheduled
@@ -171,11 +172,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     const uint32_t tmem_base = *tmem_holder;
 
     constexpr int TILE_M = BM * CG;
-    const int num_m = (M + TILE_M - 1) / TILE_M, num_n = (N + BN - 1) / BN;
-    const int num_tiles = num_m * num_n;
+    const int num_m = (M + TILE_M - 1) / TILE_M;
+    const int num_nb = (N + BNS - 1) / BNS;                     // column blocks of one sub-tile's width
+    // Work items. NSUB = 1: one item per tile, along N first, then the next block of rows (banded orders were
+    // measured: no difference on the benchmark shapes, hot or cold L2). NSUB = 2: every block of rows is covered by
+    // wide_per_row wide items (two column blocks side by side, sharing A) followed by narrow items (one column
+    // block) for the rest; all wide items come first in the list, then all narrow ones, and item i belongs to CTA
+    // group i mod groups. The host picks wide_per_row so that the groups end up with equal work (e.g. 18 x 12 column
+    // blocks on 74 pairs: 4 wide + 4 narrow per row block give 72 pairs one wide and one narrow item each).
+    const int wide = NSUB == 2 ? wide_per_row : 0;
+    const int narrow = NSUB == 2 ? num_nb - 2 * wide : num_nb;
+    const int num_wide = num_m * wide;
+    const int num_tiles = num_wide + num_m * narrow;
+    const int wide_div = wide > 0 ? wide : 1, narrow_div = narrow > 0 ? narrow : 1;   // (a kind that is absent is never decoded)
     const int num_kb = (K + BK - 1) / BK;
     const int first_tile = blockIdx.x / CG, tile_step = gridDim.x / CG;
-    // Work list of this CTA group: whole tiles first_tile, first_tile + tile_step, ... below tiles_whole, then
+    // Work list of this CTA group: whole items first_tile, first_tile + tile_step, ... below tiles_whole, then
     // (K-split) part unit_part of tile unit_tile: stages [unit_sb, unit_se) of its k-loop.
     const int num_kstages = (num_kb + KBS - 1) / KBS;
     const int tiles_whole = num_tiles - split_tiles;
@@ -184,10 +196,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     const int unit_tile = tiles_whole + unit_slot;
     const int unit_sb = has_unit ? num_kstages * unit_part / split_s : 0;
     const int unit_se = has_unit ? num_kstages * (unit_part + 1) / split_s : 0;
-    // Tile order: along N first, then the next block of rows (banded orders were measured: no difference on the
-    // benchmark shapes, hot or cold L2). A wave of concurrent tiles then shares a few row blocks of A.
-    auto tile_n = [&](int t) { return t % num_n; };
-    auto tile_m = [&](int t) { return t / num_n; };
+    struct Item { int m0, n0, nsub; };                          // first row (of the pair), first column, sub-tiles
+    auto item = [&](int t) -> Item {
+        if (NSUB == 2 && t < num_wide) return Item{(t / wide_div) * TILE_M, (t % wide_div) * 2 * BNS, 2};
+        const int u = t - num_wide;
+        return Item{(u / narrow_div) * TILE_M, (2 * wide + u % narrow_div) * BNS, 1};
+    };
+    // items of this group below L
+    auto count_below = [&](int L) { return L > first_tile ? (L - first_tile + tile_step - 1) / tile_step : 0; };
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer (both CTAs of a pair)
         // The kernel is always launched so that it may start while the kernel ahead of it in the stream is finishing
@@ -212,8 +228,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         bool ok = true;
         bool withhold = rc.starve != 0;                     // test hook: this CTA's very first stage never arrives
         auto produce = [&](int t, int sb, int se) {
-            const int m0 = tile_m(t) * TILE_M + rank * BM;
-            const int n0 = tile_n(t) * BN + rank * L::B_ROWS;
+            const Item it = item(t);
+            const int m0 = it.m0 + rank * BM;
+            const int n0 = it.n0 + rank * L::B_ROWS;
+            const int nsub = it.nsub;
+            const uint32_t kb_bytes = L::A_BYTES + nsub * L::B_BYTES;
             if (lane == 0) {
                 const uint64_t keep = l2_policy_evict_last();        // operands are re-read by other tiles: keep them in L2
                 for (int ks = sb; ks < se; ++ks) {
@@ -234,18 +253,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                         const int kx = (kb + sub) * BK;
                         if (CG == 2) {
                             // the leader's barrier counts the bytes of both CTAs
-                            if (leader) mbar_arrive_expect_tx(full_bar(stage, sub), 2 * L::KB_BYTES);
+                            if (leader) mbar_arrive_expect_tx(full_bar(stage, sub), 2 * kb_bytes);
                             const uint32_t fb = mapa_shared(full_bar(stage, sub), 0);
                             tma_load_2d_pair_hint(sa, &tm_a, fb, kx, m0, keep);
 #pragma unroll
                             for (int h = 0; h < NSUB; ++h)
-                                tma_load_2d_pair_hint(sa + L::A_BYTES + h * L::B_BYTES, &tm_b, fb, kx, n0 + h * BNS, keep);
+                                if (h < nsub) tma_load_2d_pair_hint(sa + L::A_BYTES + h * L::B_BYTES, &tm_b, fb, kx, n0 + h * BNS, keep);
                         } else {
-                            mbar_arrive_expect_tx(full_bar(stage, sub), L::KB_BYTES);
+                            mbar_arrive_expect_tx(full_bar(stage, sub), kb_bytes);
                             tma_load_2d_hint(sa, &tm_a, full_bar(stage, sub), kx, m0, keep);
 #pragma unroll
                             for (int h = 0; h < NSUB; ++h)
-                                tma_load_2d_hint(sa + L::A_BYTES + h * L::B_BYTES, &tm_b, full_bar(stage, sub), kx, n0 + h * BNS, keep);
+                                if (h < nsub) tma_load_2d_hint(sa + L::A_BYTES + h * L::B_BYTES, &tm_b, full_bar(stage, sub), kx, n0 + h * BNS, keep);
                         }
                     }
                     ++issued;
@@ -306,6 +325,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             // the stage is free (in both CTAs) once the MMAs issued so far have read it. One commit per stage, not per
             // k-block: with 128-byte stages the commits and barrier round trips cost ~8% of the run time
             auto release_stage = [&](int st) {
+                // (signalling only the leader and letting its producer pass the release on to the peer with a remote
+                // arrive was measured: 147 against 110 us on the MLP down-projection. The release -> refill latency
+                // is what this pipeline lives on.)
                 if (CG == 2) { tc_commit_pair(empty_bar(st)); tc_commit_pair(mapa_shared(empty_bar(st), 1)); }
                 else tc_commit(empty_bar(st));
             };
@@ -313,9 +335,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 if (CG == 2) { tc_commit_pair(tfull_bar(cc & 1)); tc_commit_pair(mapa_shared(tfull_bar(cc & 1), 1)); }
                 else tc_commit(tfull_bar(cc & 1));
             };
-            auto mma_tile = [&](int sb, int se) {
+            auto mma_tile = [&](int nsub, int sb, int se) {
                 int ks = sb;
-                if (NSUB == 2) {
+                if (NSUB == 2 && nsub == 2) {
                     // Staggered start. Both slots were published together, but the epilogue drains slot 0 first:
                     // sub-tile 0 runs ahead over the stages the ring can hold while slot 1 is still being drained,
                     // then sub-tile 1 catches up on the same stages and hands them back.
@@ -350,18 +372,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                         if (!wait_full(stage, sub, phase)) { ok = false; break; }
 #pragma unroll
                         for (int h = 0; h < NSUB; ++h)
-                            issue(stage, sub, ks * KBS + sub, h, slot_tmem(c + h), ks == sb && sub == 0);
+                            if (h < nsub) issue(stage, sub, ks * KBS + sub, h, slot_tmem(c + h), ks == sb && sub == 0);
                     }
                     if (!ok) return;
                     release_stage(stage);
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
 #pragma unroll
-                for (int h = 0; h < NSUB; ++h) publish(c + h);
-                c += NSUB;
+                for (int h = 0; h < NSUB; ++h)
+                    if (h < nsub) publish(c + h);
+                c += nsub;
             };
-            for (int t = first_tile; t < tiles_whole && ok; t += tile_step) mma_tile(0, num_kstages);
-            if (has_unit && ok) mma_tile(unit_sb, unit_se);
+            for (int t = first_tile; t < tiles_whole && ok; t += tile_step) mma_tile((NSUB == 2 && t < num_wide) ? 2 : 1, 0, num_kstages);
+            if (has_unit && ok) mma_tile(1, unit_sb, unit_se);
         }
     } else {
         // ------------------------------------------------------------ epilogue (warps 2..5, helpers 6..9)
@@ -377,8 +400,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         const uint32_t staging = base + stg_off;
         uint8_t* staging_ptr = base_ptr + stg_off;
         // The epilogue of a CTA's last tile overlaps with nothing: there the helpers take the upper part of the boxes.
-        const int n_regular = tiles_whole > first_tile ? (tiles_whole - first_tile + tile_step - 1) / tile_step : 0;
-        const int n_sub = n_regular * NSUB;            // sub-tiles of whole tiles this CTA works on
+        const int n_regular = count_below(tiles_whole);                              // whole items of this CTA group
+        const int n_sub = n_regular + count_below(min(num_wide, tiles_whole));      // their sub-tiles (a wide item has two)
+        const int t_last = first_tile + (n_regular - 1) * tile_step;                // the group's last whole item
+        const int last_nsub = (NSUB == 2 && n_regular > 0 && t_last < num_wide) ? 2 : 1;
         constexpr int ALL_CHUNKS = BNS / 32;
         constexpr int C_SPLIT = 2 * (BNS / 64 - BNS / 128);          // 32-column chunks the epilogue warps keep on that tile
         const bool helpers_on = !RAW_I32 && n_regular > 0 && !has_unit && C_SPLIT < ALL_CHUNKS;
@@ -391,7 +416,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         // chunks [c_lo, c_hi) of sub-tile h of tile t; `shared_tile`: the helpers work on this sub-tile too
         auto epi_tile = [&](int t, int h, bool unit, int c_lo, int c_hi, bool shared_tile) {
             const int buf = c & 1;
-            const int m0 = tile_m(t) * TILE_M + rank * BM, n0 = tile_n(t) * BN + h * BNS;
+            const Item it = item(t);
+            const int m0 = it.m0 + rank * BM, n0 = it.n0 + h * BNS;
             const float* sch_buf = sm_sch + buf * BNS;
             const float* bias_buf = sm_bias + buf * BNS;
             if (!RAW_I32 && !helper) {
@@ -416,6 +442,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             // One chunk = 32 accumulator columns of this thread's row. Two chunks make a 32 x 64 output box.
             // The TMEM load of the next chunk is in flight while the current one is converted.
             const uint64_t st2 = pack2(st, st);
+            // optional side output: the largest magnitude this thread's row receives from this sub-tile (bf16 values as
+            // stored; columns outside N come out as +0 and do not count), merged into rowmax[row] at the end
+            __nv_bfloat162 rmax2 = __float2bfloat162_rn(0.f);
+            auto flush_rowmax = [&]() {
+                if (RAW_I32 || rowmax == nullptr || row >= M) return;
+                const uint32_t mb = *reinterpret_cast<const uint32_t*>(&rmax2);
+                const uint32_t bits = max(mb << 16, mb & 0xffff0000u);      // non-negative floats order like their bit patterns
+                if (bits != 0u) atomicMax(reinterpret_cast<unsigned int*>(rowmax) + row, bits);
+            };
             auto process = [&](int cc, const uint32_t (&v)[32]) {
                 const int col = cc * 32, hh = cc & 1, cb = cc >> 1;
                 const int sbuf = cb & (L::STAGING_BUFS - 1);  // staging boxes alternate: the store of one overlaps the next
@@ -444,6 +479,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                         a1 = __fadd_rn(a1, bi.y);
                     }
                     packed[j] = pack_bf16x2(a0, a1);
+                }
+                if (rowmax != nullptr) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) rmax2 = __hmax2(rmax2, __habs2(*reinterpret_cast<const __nv_bfloat162*>(&packed[j])));
                 }
                 if (hh == 0) {
                     // the store issued STAGING_BUFS boxes ago (same staging box) must have finished reading it
@@ -489,6 +528,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     else release_accumulator();
                     process(cc + 1, vb);
                 }
+                flush_rowmax();
                 return;
             }
             // ---- one K part of a split tile. Every part adds its int32 accumulators into the tile's slab in
@@ -536,21 +576,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 for (int j = 0; j < 32; ++j) va[j] = static_cast<uint32_t>(sm_slab[(cc * 32 + j) * BM]);
                 process(cc, va);
             }
+            flush_rowmax();
         };
         if (!helper) {
             for (int t = first_tile; t < tiles_whole; t += tile_step) {
-#pragma unroll
-                for (int h = 0; h < NSUB; ++h, ++c) {
-                    const bool shared_tile = helpers_on && c >= n_sub - NSUB;
+                const int nsub = (NSUB == 2 && t < num_wide) ? 2 : 1;
+                for (int h = 0; h < nsub; ++h, ++c) {
+                    const bool shared_tile = helpers_on && c >= n_sub - last_nsub;
                     epi_tile(t, h, false, 0, shared_tile ? C_SPLIT : ALL_CHUNKS, shared_tile);
                 }
             }
             if (has_unit) epi_tile(unit_tile, 0, true, 0, ALL_CHUNKS, false);
         } else if (helpers_on) {
-            const int t_last = first_tile + (n_regular - 1) * tile_step;
-            c = n_sub - NSUB;
-#pragma unroll
-            for (int h = 0; h < NSUB; ++h, ++c) epi_tile(t_last, h, false, C_SPLIT, ALL_CHUNKS, true);
+            c = n_sub - last_nsub;
+            for (int h = 0; h < last_nsub; ++h, ++c) epi_tile(t_last, h, false, C_SPLIT, ALL_CHUNKS, true);
         }
         if (!RAW_I32 && lane == 0) bulk_wait_group<0>();
     }
@@ -608,14 +647,16 @@ struct TcConfig {
 };
 constexpr TcConfig kConfigs[] = {
     // measured on the c4 shapes (hot L2): pair 256x256 3 x 256 B: 115 / 111 us; one CTA 128x256 4 x 128 B: 129 / 121 us;
-    // pair 256x192: 130 / 123 us; one CTA 128x128: 164 / 154 us; pair 256x128: 168 / 162 us
+    // pair 256x192: 130 / 123 us; one CTA 128x128: 164 / 154 us; pair 256x128: 168 / 162 us. Stage shapes of the
+    // 256x256 pair at the same 192 KB: 6 x 128 B of K 126 / 118 us, 2 x 384 B 123 / 117 us (both directions lose).
+    // Pair tiles of two sub-tiles: 2 x 256 wins where K is deep and the wide items fill whole waves (M = 9472,
+    // K = 12288 -> N = 3072: 213-225 against 230-237 us); 2 x 192 lost everywhere (N = 192 MMAs) and is not built.
     {"tc 128x256 per CTA, 4 stages x 128 B of K", 1, 256, 1, 4, 1, 0.89f},
     {"tc 128x128 per CTA, 3 stages x 256 B of K", 1, 128, 1, 3, 2, 0.72f},
     {"tc 256x256 per CTA pair, 3 stages x 256 B of K", 2, 256, 1, 3, 2, 1.00f},
     {"tc 256x128 per CTA pair, 4 stages x 256 B of K", 2, 128, 1, 4, 2, 0.70f},
     {"tc 256x192 per CTA pair, 3 stages x 256 B of K", 2, 192, 1, 3, 2, 0.88f},
-    {"tc 256x384 (2 x 192) per CTA pair, 4 stages x 128 B of K", 2, 192, 2, 4, 1, 1.05f},
-    {"tc 256x512 (2 x 256) per CTA pair, 4 stages x 128 B of K", 2, 256, 2, 4, 1, 1.05f},
+    {"tc 256x512 (2 x 256) per CTA pair, 4 stages x 128 B of K", 2, 256, 2, 4, 1, 1.08f},
 };
 constexpr int kNumConfigs = sizeof(kConfigs) / sizeof(kConfigs[0]);
 constexpr int kNoSplitBit = 0x100;        // added to a forced configuration id: no K-split of the partial wave
@@ -669,7 +710,7 @@ int launch_cfg(const GemmArgs& a, const TcPlan& plan, cudaStream_t st) {
                                        RAW ? static_cast<int32_t*>(a.out) : nullptr, a.M, a.N, a.K, rc,
                                        plan.split_tiles, plan.split_parts,
                                        reinterpret_cast<int32_t*>(static_cast<uint8_t*>(a.split_ws) + kCounterBytes),
-                                       static_cast<int*>(a.split_ws));
+                                       static_cast<int*>(a.split_ws), plan.wide_per_row, a.raw_i32 ? nullptr : a.rowmax);
     return e == cudaSuccess ? W8A8_OK : W8A8_ERR_CUDA;
 }
 
@@ -681,8 +722,7 @@ int launch_by_id(const GemmArgs& a, const TcPlan& plan, cudaStream_t st) {
         case 2: return launch_cfg<2, 256, 1, 3, 2, RAW>(a, plan, st);
         case 3: return launch_cfg<2, 128, 1, 4, 2, RAW>(a, plan, st);
         case 4: return launch_cfg<2, 192, 1, 3, 2, RAW>(a, plan, st);
-        case 5: return launch_cfg<2, 192, 2, 4, 1, RAW>(a, plan, st);
-        case 6: return launch_cfg<2, 256, 2, 4, 1, RAW>(a, plan, st);
+        case 5: return launch_cfg<2, 256, 2, 4, 1, RAW>(a, plan, st);
         default: return W8A8_ERR_INVALID_ARG;
     }
 }
@@ -693,30 +733,59 @@ int launch_by_id(const GemmArgs& a, const TcPlan& plan, cudaStream_t st) {
 // kMinStagesPerPart pipeline stages per part, at most kMaxSplit parts, and only if the scratch has room),
 // which shortens it to 1/parts of a tile time plus the cost of adding the partial sums up. With only_if_faster
 // the cut is dropped when the estimate says it does not pay (it pays for deep K: K >= ~8192).
-TcPlan plan_config(int id, int M, int N, int K, bool allow_split, bool only_if_faster, size_t scratch_bytes, double* est_us) {
+// Configurations of two sub-tiles are never cut; their degree of freedom is how many of a row block's column
+// blocks are paired into wide items (see the kernel): the count that gives the busiest group the least work wins.
+TcPlan plan_config(int id, int M, int N, int K, bool allow_split, bool only_if_faster, size_t scratch_bytes, int wide_forced,
+                   double* est_us) {
     const TcConfig& c = kConfigs[id];
     TcPlan p{};
     p.config = id;
     const int max_groups = sm_count() / c.cg;
-    const int bn = c.bns * c.nsub;
-    const long tiles = static_cast<long>((M + BM * c.cg - 1) / (BM * c.cg)) * ((N + bn - 1) / bn);
+    const int num_m = (M + BM * c.cg - 1) / (BM * c.cg);
+    const double fixed_us = 4.0;                       // launch, pipeline fill, last epilogue
+    if (c.nsub == 2) {
+        // ~20.3 int8 TOPS per SM for the 256 x 256 pair tile in whole waves; a unit = one column block of a row block
+        const int num_nb = (N + c.bns - 1) / c.bns;
+        const double unit_us = 2.0 * BM * c.bns * static_cast<double>(K) / 20.3e6;
+        const double wide_unit_us = unit_us / c.eff, narrow_unit_us = unit_us / 0.88;   // narrow items run on four 128-byte stages
+        const double wide_exposed_us = 2.5;            // the drain of a wide item's first accumulator overlaps nothing
+        int best_w = 0;
+        double best = 0.0;
+        for (int w = (wide_forced >= 0 ? wide_forced : 0); w <= (wide_forced >= 0 ? wide_forced : num_nb / 2); ++w) {
+            const long wide_items = static_cast<long>(num_m) * w, all_items = wide_items + static_cast<long>(num_m) * (num_nb - 2 * w);
+            const long groups = all_items < max_groups ? all_items : max_groups;
+            double worst = 0.0;
+            for (long g = 0; g < groups; ++g) {
+                const long nw = wide_items > g ? (wide_items - g + groups - 1) / groups : 0;
+                const long na = all_items > g ? (all_items - g + groups - 1) / groups : 0;
+                const double t = nw * (2.0 * wide_unit_us + wide_exposed_us) + (na - nw) * narrow_unit_us;
+                if (t > worst) worst = t;
+            }
+            if (w == (wide_forced >= 0 ? wide_forced : 0) || worst < best) { best = worst; best_w = w; }
+        }
+        const long items = static_cast<long>(num_m) * (num_nb - best_w);
+        p.wide_per_row = best_w;
+        p.groups = static_cast<int>(items < max_groups ? items : max_groups);
+        if (est_us) *est_us = fixed_us + best;
+        return p;
+    }
+    const long tiles = static_cast<long>(num_m) * ((N + c.bns - 1) / c.bns);
+    const int bn = c.bns;
     const int whole_waves = static_cast<int>(tiles / max_groups);
     const int rest = static_cast<int>(tiles % max_groups);
     const int kstages = ((K + BK - 1) / BK + c.kbs - 1) / c.kbs;
     int parts = 1;
-    if (allow_split && rest > 0 && c.nsub == 1) {      // tiles of two sub-tiles are never cut
+    if (allow_split && rest > 0) {
         parts = max_groups / rest;
         if (parts > kstages / kMinStagesPerPart) parts = kstages / kMinStagesPerPart;
         if (parts > kMaxSplit) parts = kMaxSplit;
         const size_t need = kCounterBytes + static_cast<size_t>(rest) * c.cg * bn * BM * sizeof(int32_t);
         if (parts < 2 || need > scratch_bytes) parts = 1;
     }
-    // ~20.3 int8 TOPS per SM for configuration 2 in whole waves. A partial wave that is left whole runs its
-    // tiles faster than that (measured ~0.72 of the tile time with few SMs active: the operand traffic of a full
-    // wave is what holds the rate down); a wave cut along K keeps every SM busy and pays ~10 us for zeroing the
-    // slabs, the reductions, the pipeline refill and the read-back.
+    // A partial wave that is left whole runs its tiles faster than the full-wave rate (measured ~0.72 of the tile
+    // time with few SMs active: the operand traffic of a full wave is what holds the rate down); a wave cut along K
+    // keeps every SM busy and pays ~10 us for zeroing the slabs, the reductions, the pipeline refill and the read-back.
     const double tile_us = 2.0 * BM * bn * static_cast<double>(K) / 20.3e6 / c.eff;
-    const double fixed_us = 4.0;                       // launch, pipeline fill, last epilogue
     const double whole_rest_us = tile_us * (0.72 + 0.28 * rest / max_groups);
     const double split_rest_us = tile_us / parts + 10.0;
     if (parts > 1 && only_if_faster && split_rest_us >= whole_rest_us) parts = 1;
@@ -743,17 +812,25 @@ int tc_num_configs() { return kNumConfigs; }
 const char* tc_config_name(int id) { return (id >= 0 && id < kNumConfigs) ? kConfigs[id].name : nullptr; }
 
 TcPlan tc_plan(int M, int N, int K, int forced, size_t scratch_bytes) {
-    // forced: -1 automatic, -2 automatic without K-split, id, or id + 0x100 for that configuration without K-split
+    // forced: -1 automatic, -2 automatic without K-split, id, or id + 0x100 for that configuration without K-split;
+    // bits 12-19, if not zero, are 1 + the number of wide items per row block (two-sub-tile configurations)
     const bool allow_split = forced == -1 || (forced >= 0 && (forced & kNoSplitBit) == 0);
     const int id = forced < 0 ? -1 : (forced & (kNoSplitBit - 1));
-    if (id >= 0 && id < kNumConfigs) return plan_config(id, M, N, K, allow_split, false, scratch_bytes, nullptr);   // forced: cut whenever possible
+    const int wide_forced = forced < 0 ? -1 : ((forced >> 12) & 0xff) - 1;
+    if (id >= 0 && id < kNumConfigs) {
+        int wf = wide_forced;
+        if (kConfigs[id].nsub == 2 && wf > ((N + kConfigs[id].bns - 1) / kConfigs[id].bns) / 2) wf = -1;   // not possible: choose
+        return plan_config(id, M, N, K, allow_split, false, scratch_bytes, wf, nullptr);   // forced: cut whenever possible
+    }
     // lowest estimated time; on (near) ties the earlier entry of this preference order wins
-    constexpr int order[] = {2, 0, 4, 3, 1};
+    constexpr int order[] = {2, 5, 0, 4, 3, 1};
     TcPlan best{};
     double best_us = 0.0;
     for (int i = 0; i < static_cast<int>(sizeof(order) / sizeof(order[0])); ++i) {
+        // wide tiles expose one accumulator drain per item: measured to pay only where the k-loop is long
+        if (kConfigs[order[i]].nsub == 2 && K < 8192) continue;
         double us = 0.0;
-        const TcPlan p = plan_config(order[i], M, N, K, allow_split, true, scratch_bytes, &us);
+        const TcPlan p = plan_config(order[i], M, N, K, allow_split, true, scratch_bytes, -1, &us);
         if (i == 0 || us < best_us * 0.97) { best = p; best_us = us; }
     }
     return best;

@@ -66,8 +66,9 @@ int* sticky_status_word();
 // ---- quantize.cu
 // status_to_clear: workspace status word the kernel resets (or nullptr).
 // mult: per-input-channel factors fp32 [K] multiplied into the operand first (SmoothQuant hook), or nullptr.
-cudaError_t launch_quantize_bf16(const void* A, int64_t lda, int M, int K, const float* mult, int8_t* qa, float* s_tok,
-                                 int* status_to_clear, cudaStream_t st);
+// amax: the absmax of every row fp32 [M] handed in by the producer of A (one-pass quantizer), or nullptr; not with mult.
+cudaError_t launch_quantize_bf16(const void* A, int64_t lda, int M, int K, const float* mult, const float* amax, int8_t* qa,
+                                 float* s_tok, int* status_to_clear, cudaStream_t st);
 cudaError_t launch_quantize_f32(const float* W, int64_t ldw, int N, int K, const float* mult, int8_t* qw, float* s_ch,
                                 cudaStream_t st);
 
@@ -86,6 +87,7 @@ struct GemmArgs {
     int* status;           // workspace status word
     bool after_quantizer;  // launched behind the quantizer with programmatic dependent launch
     void* split_ws;        // scratch of the K-split (counters, then partial accumulators), or nullptr
+    float* rowmax;         // fp32 [M], zero at launch: receives max_n |out[m,n]| of the bf16 values written; or nullptr
 };
 cudaError_t launch_gemm_simt(const GemmArgs& a, cudaStream_t st);
 
@@ -99,8 +101,10 @@ struct TcPlan {
     int split_tiles;       // tiles of the partial wave that are cut along K
     int split_parts;       // parts per such tile
     size_t scratch_bytes;  // scratch the split needs (counters, then one int32 slab per tile); all zero at launch
+    int wide_per_row;      // configurations of two sub-tiles: wide items (two column blocks) per block of rows
 };
-// Picks a configuration for the shape (or `forced` if >= 0; forced + 0x100 = that configuration without K-split).
+// Picks a configuration for the shape (or `forced` if >= 0; forced + 0x100 = that configuration without K-split;
+// bits 12-19 of `forced`, if not zero, are 1 + the number of wide items per block of rows).
 // A split is planned only if its scratch fits in scratch_bytes.
 TcPlan tc_plan(int M, int N, int K, int forced, size_t scratch_bytes);
 // Scratch the automatic choice uses when it is given enough.

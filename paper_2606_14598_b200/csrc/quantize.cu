@@ -174,11 +174,13 @@ __device__ __forceinline__ void bulk_load_row(uint32_t smem_dst, const void* gsr
 
 // WPR consumer warps share a row (power of two <= SG_WARPS); a stage holds RPS = SG_WARPS / WPR rows.
 // SMOOTH: multiply every element by mult[k] first (SmoothQuant hook).
-template <int WPR, bool SMOOTH>
+// GIVEN: the absmax of every row is handed in (amax_in, written by the producer of the activations, possibly the
+// kernel just ahead in the stream): the search pass and the exchange between the row's warps fall away.
+template <int WPR, bool SMOOTH, bool GIVEN>
 __global__ void __launch_bounds__(SG_THREADS, 2)
 quant_rows_staged_kernel(const __nv_bfloat16* __restrict__ x, int64_t ld, int rows, int K,
                          int8_t* __restrict__ q, float* __restrict__ s_out, const QuantCtl qc, int num_stages,
-                         const float* __restrict__ mult) {
+                         const float* __restrict__ mult, const float* amax_in) {
     int* const status = qc.status;
     // a dependent kernel (the GEMM) may set itself up while this one runs; it waits for this grid before reading
     grid_dep_launch_dependents();
@@ -250,7 +252,10 @@ quant_rows_staged_kernel(const __nv_bfloat16* __restrict__ x, int64_t ld, int ro
             const bool live = ok && row < rows;
             const uint4* srow = reinterpret_cast<const uint4*>(base_ptr + stage * stage_bytes + slot * row_bytes);
             float amax = 0.f;
-            if (SMOOTH) {
+            if (GIVEN) {
+                // plain (coherent) load: the value may have been written by the kernel ahead while this one was resident
+                if (row < rows) amax = __ldcg(amax_in + row);
+            } else if (SMOOTH) {
                 if (live) {
 #pragma unroll 2
                     for (int u = part * 32 + lane; u < units; u += WPR * 32) {
@@ -267,9 +272,11 @@ quant_rows_staged_kernel(const __nv_bfloat16* __restrict__ x, int64_t ld, int ro
                 }
                 amax = unpack_max(m2);
             }
+            if (!GIVEN) {
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-            if (WPR > 1) {
+                for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+            }
+            if (WPR > 1 && !GIVEN) {
                 // the WPR warps of a row exchange their partial maxima through shared memory
                 if (lane == 0) s_red[warp] = amax;
                 asm volatile("bar.sync %0, %1;" ::"r"(1 + slot), "n"(WPR * 32) : "memory");
@@ -371,10 +378,11 @@ template <> struct Chunk<float> {
 // WPR warps per row (a power of two <= 16); a CTA works on RPC = 16 / WPR rows at a time. Rows with more
 // than WPR*32*CPL chunks stream the surplus twice (absmax pass, then quantize pass) from memory / L2.
 // SMOOTH (SmoothQuant hook): elements are widened to fp32 and multiplied by mult[k] as they are loaded.
-template <typename T, int WPR, bool SMOOTH>
+template <typename T, int WPR, bool SMOOTH, bool GIVEN>
 __global__ void __launch_bounds__(WARPS * 32, 1)
 quant_rows_kernel(const T* __restrict__ x, int64_t ld, int rows, int K,
-                  int8_t* __restrict__ q, float* __restrict__ s_out, int* status, const float* __restrict__ mult) {
+                  int8_t* __restrict__ q, float* __restrict__ s_out, int* status, const float* __restrict__ mult,
+                  const float* amax_in) {
     using C = Chunk<typename std::conditional<SMOOTH, float, T>::type>;
     auto fetch = [&](C& c, const T* row, int chunk) {
         c.load(row + chunk * 16);
@@ -404,22 +412,26 @@ quant_rows_kernel(const T* __restrict__ x, int64_t ld, int rows, int K,
             const int c = c0 + i * STRIDE;
             if (live && c < nchunks) fetch(reg[i], xr, c); else reg[i].zero();
         }
+        if (GIVEN) {
+            if (live) amax = __ldcg(amax_in + row);
+        } else {
 #pragma unroll
-        for (int i = 0; i < CPL; ++i) amax = fmaxf(amax, reg[i].absmax());
-        if (live) {
-            for (int c = c0 + CPL * STRIDE; c < nchunks; c += STRIDE) {   // surplus chunks (very long rows)
-                C t;
-                fetch(t, xr, c);
-                amax = fmaxf(amax, t.absmax());
+            for (int i = 0; i < CPL; ++i) amax = fmaxf(amax, reg[i].absmax());
+            if (live) {
+                for (int c = c0 + CPL * STRIDE; c < nchunks; c += STRIDE) {   // surplus chunks (very long rows)
+                    C t;
+                    fetch(t, xr, c);
+                    amax = fmaxf(amax, t.absmax());
+                }
             }
-        }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-        if (WPR > 1) {
-            if (lane == 0) s_red[warp] = amax;
-            __syncthreads();
+            for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+            if (WPR > 1) {
+                if (lane == 0) s_red[warp] = amax;
+                __syncthreads();
 #pragma unroll
-            for (int w = 0; w < WPR; ++w) amax = fmaxf(amax, s_red[slot * WPR + w]);
+                for (int w = 0; w < WPR; ++w) amax = fmaxf(amax, s_red[slot * WPR + w]);
+            }
         }
         if (live) {
             const RowScale s = make_row_scale(amax);
@@ -436,7 +448,7 @@ quant_rows_kernel(const T* __restrict__ x, int64_t ld, int rows, int K,
                 *reinterpret_cast<uint4*>(qr + c * 16) = t.quantize(s);
             }
         }
-        if (WPR > 1) __syncthreads();    // s_red may be rewritten by the next sweep
+        if (WPR > 1 && !GIVEN) __syncthreads();    // s_red may be rewritten by the next sweep
     }
 }
 
@@ -459,33 +471,37 @@ cudaError_t launch_pdl(void (*kern)(KArgs...), int grid, int block, size_t smem,
     return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
 }
 
+// amax: the rows' absmax handed in (one pass), or nullptr (the kernel searches for it). Not combined with mult.
 template <typename T, int WPR>
 cudaError_t launch_reg(const T* x, int64_t ld, int rows, int K, int8_t* q, float* s, int* status, const float* mult,
-                       cudaStream_t st) {
+                       const float* amax, cudaStream_t st) {
     constexpr int RPC = WARPS / WPR;
     const int units = (rows + RPC - 1) / RPC;
     const int cap = sm_count() * 2;
     const int grid = units < cap ? units : cap;
-    const float* no_mult = nullptr;
-    if (mult != nullptr) return launch_pdl(quant_rows_kernel<T, WPR, true>, grid, WARPS * 32, 0, st, x, ld, rows, K, q, s, status, mult);
-    return launch_pdl(quant_rows_kernel<T, WPR, false>, grid, WARPS * 32, 0, st, x, ld, rows, K, q, s, status, no_mult);
+    const float* none = nullptr;
+    if (amax != nullptr)
+        return launch_pdl(quant_rows_kernel<T, WPR, false, true>, grid, WARPS * 32, 0, st, x, ld, rows, K, q, s, status, none, amax);
+    if (mult != nullptr)
+        return launch_pdl(quant_rows_kernel<T, WPR, true, false>, grid, WARPS * 32, 0, st, x, ld, rows, K, q, s, status, mult, none);
+    return launch_pdl(quant_rows_kernel<T, WPR, false, false>, grid, WARPS * 32, 0, st, x, ld, rows, K, q, s, status, none, none);
 }
 
 template <typename T>
 cudaError_t dispatch_reg(const T* x, int64_t ld, int rows, int K, int8_t* q, float* s, int* status, const float* mult,
-                         cudaStream_t st) {
+                         const float* amax, cudaStream_t st) {
     const int nchunks = K / 16;
     // fewest warps per row that keep the whole row in registers (<= CPL chunks per lane)
-    if (nchunks <= 32 * CPL)  return launch_reg<T, 1>(x, ld, rows, K, q, s, status, mult, st);
-    if (nchunks <= 64 * CPL)  return launch_reg<T, 2>(x, ld, rows, K, q, s, status, mult, st);
-    if (nchunks <= 128 * CPL) return launch_reg<T, 4>(x, ld, rows, K, q, s, status, mult, st);
-    if (nchunks <= 256 * CPL) return launch_reg<T, 8>(x, ld, rows, K, q, s, status, mult, st);
-    return launch_reg<T, 16>(x, ld, rows, K, q, s, status, mult, st);
+    if (nchunks <= 32 * CPL)  return launch_reg<T, 1>(x, ld, rows, K, q, s, status, mult, amax, st);
+    if (nchunks <= 64 * CPL)  return launch_reg<T, 2>(x, ld, rows, K, q, s, status, mult, amax, st);
+    if (nchunks <= 128 * CPL) return launch_reg<T, 4>(x, ld, rows, K, q, s, status, mult, amax, st);
+    if (nchunks <= 256 * CPL) return launch_reg<T, 8>(x, ld, rows, K, q, s, status, mult, amax, st);
+    return launch_reg<T, 16>(x, ld, rows, K, q, s, status, mult, amax, st);
 }
 
 template <int WPR>
 cudaError_t launch_staged(const __nv_bfloat16* x, int64_t ld, int rows, int K, int8_t* q, float* s, int* status,
-                          const float* mult, cudaStream_t st) {
+                          const float* mult, const float* amax, cudaStream_t st) {
     constexpr int RPS = SG_WARPS / WPR;
     const int stage_bytes = RPS * K * 2;
     const int groups = (rows + RPS - 1) / RPS;
@@ -501,43 +517,48 @@ cudaError_t launch_staged(const __nv_bfloat16* x, int64_t ld, int rows, int K, i
     const int smem = num_stages * stage_bytes + 16 * num_stages + SG_WARPS * 4 + 16 + 128;
     static PerDeviceOnce smem_opt_in;
     const cudaError_t attr_err = smem_opt_in.run([] {
-        cudaError_t e = cudaFuncSetAttribute(quant_rows_staged_kernel<WPR, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(quant_rows_staged_kernel<WPR, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              SG_SMEM_MAX);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(quant_rows_staged_kernel<WPR, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            e = cudaFuncSetAttribute(quant_rows_staged_kernel<WPR, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     SG_SMEM_MAX);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(quant_rows_staged_kernel<WPR, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      SG_SMEM_MAX);
         return e;
     });
     if (attr_err != cudaSuccess) return attr_err;
     const int cap = ctas_per_sm * sm_count();
     const int grid = groups < cap ? groups : cap;
-    const float* no_mult = nullptr;
+    const float* none = nullptr;
     const QuantCtl qc{status, sticky_status_word(), wait_limit_ns(), starve_mode() == kStarveQuant ? 1 : 0};
+    if (amax != nullptr)
+        return launch_pdl(quant_rows_staged_kernel<WPR, false, true>, grid, SG_THREADS, smem, st, x, ld, rows, K, q, s, qc, num_stages, none, amax);
     if (mult != nullptr)
-        return launch_pdl(quant_rows_staged_kernel<WPR, true>, grid, SG_THREADS, smem, st, x, ld, rows, K, q, s, qc, num_stages, mult);
-    return launch_pdl(quant_rows_staged_kernel<WPR, false>, grid, SG_THREADS, smem, st, x, ld, rows, K, q, s, qc, num_stages, no_mult);
+        return launch_pdl(quant_rows_staged_kernel<WPR, true, false>, grid, SG_THREADS, smem, st, x, ld, rows, K, q, s, qc, num_stages, mult, none);
+    return launch_pdl(quant_rows_staged_kernel<WPR, false, false>, grid, SG_THREADS, smem, st, x, ld, rows, K, q, s, qc, num_stages, none, none);
 }
 
 } // namespace
 
-cudaError_t launch_quantize_bf16(const void* A, int64_t lda, int M, int K, const float* mult, int8_t* qa, float* s_tok,
-                                 int* status_to_clear, cudaStream_t st) {
+cudaError_t launch_quantize_bf16(const void* A, int64_t lda, int M, int K, const float* mult, const float* amax, int8_t* qa,
+                                 float* s_tok, int* status_to_clear, cudaStream_t st) {
     const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(A);
     // a warp handles up to 4 KB of a row (measured best among 1-16 KB); rows of up to 64 KB (K <= 32768) go
     // through the staged kernel with several stages, rows of up to 113 KB with two stages of one row each (a warp
     // then walks up to 7 KB), longer ones through the register kernel
     const int row_bytes = K * 2;
-    if (row_bytes <= 2048)  return launch_staged<1>(x, lda, M, K, qa, s_tok, status_to_clear, mult, st);   // 16 rows per stage
-    if (row_bytes <= 8192)  return launch_staged<2>(x, lda, M, K, qa, s_tok, status_to_clear, mult, st);   // 8 rows per stage
-    if (row_bytes <= 16384) return launch_staged<4>(x, lda, M, K, qa, s_tok, status_to_clear, mult, st);
-    if (row_bytes <= 32768) return launch_staged<8>(x, lda, M, K, qa, s_tok, status_to_clear, mult, st);
-    if (2 * row_bytes + 1024 <= SG_SMEM_MAX) return launch_staged<16>(x, lda, M, K, qa, s_tok, status_to_clear, mult, st);
-    return dispatch_reg<__nv_bfloat16>(x, lda, M, K, qa, s_tok, status_to_clear, mult, st);
+    if (row_bytes <= 2048)  return launch_staged<1>(x, lda, M, K, qa, s_tok, status_to_clear, mult, amax, st);   // 16 rows per stage
+    if (row_bytes <= 8192)  return launch_staged<2>(x, lda, M, K, qa, s_tok, status_to_clear, mult, amax, st);   // 8 rows per stage
+    if (row_bytes <= 16384) return launch_staged<4>(x, lda, M, K, qa, s_tok, status_to_clear, mult, amax, st);
+    if (row_bytes <= 32768) return launch_staged<8>(x, lda, M, K, qa, s_tok, status_to_clear, mult, amax, st);
+    if (2 * row_bytes + 1024 <= SG_SMEM_MAX) return launch_staged<16>(x, lda, M, K, qa, s_tok, status_to_clear, mult, amax, st);
+    return dispatch_reg<__nv_bfloat16>(x, lda, M, K, qa, s_tok, status_to_clear, mult, amax, st);
 }
 
 cudaError_t launch_quantize_f32(const float* W, int64_t ldw, int N, int K, const float* mult, int8_t* qw, float* s_ch,
                                 cudaStream_t st) {
-    return dispatch_reg<float>(W, ldw, N, K, qw, s_ch, nullptr, mult, st);
+    return dispatch_reg<float>(W, ldw, N, K, qw, s_ch, nullptr, mult, nullptr, st);
 }
 
 } // namespace w8a8

@@ -472,6 +472,124 @@ def test_k_split_from_bf16_automatic_choice():
     assert torch.equal(out, out2)
 
 
+# ------------------------------------------------------------------------------- quantizer fused into its producer
+
+@pytest.mark.parametrize("M,K", [(1, 16), (33, 2048), (300, 3072), (40, 12288), (3, 40000), (6, 53248), (2, 66000)])
+def test_one_pass_quantizer_with_the_absmax_handed_in(M, K):
+    spec = synth.LinearSpec(f"q1p{M}x{K}", M, K, 8, outlier_frac=0.01 if K >= 256 else 0.0)
+    A = synth.make_activations(spec)
+    if M > 2:
+        A[1] = 0
+    bits = synth.bf16_bits(A)
+    rowmax = oracle.row_absmax_bf16(bits)
+    qa_ref, s_ref = oracle.quantize_act_per_token(bits)
+    # the row's own absmax: the one-pass quantizer equals the two-pass one (oracle and device)
+    qa, s = w8.int8_quantize_act_per_token_given_absmax(A.to(DEV), torch.from_numpy(rowmax).to(DEV))
+    assert np.array_equal(s.cpu().numpy().view(np.uint32), s_ref.view(np.uint32))
+    assert np.array_equal(qa.cpu().numpy(), qa_ref)
+    # a larger absmax (allowed): against the oracle's given-absmax function
+    bigger = (rowmax * np.float32(1.75) + np.float32(0.125)).astype(np.float32)
+    qa_ref2, s_ref2 = oracle.quantize_act_per_token_given_absmax(bits, bigger)
+    qa2, s2 = w8.int8_quantize_act_per_token_given_absmax(A.to(DEV), torch.from_numpy(bigger).to(DEV))
+    assert np.array_equal(s2.cpu().numpy().view(np.uint32), s_ref2.view(np.uint32))
+    assert np.array_equal(qa2.cpu().numpy(), qa_ref2)
+
+
+@pytest.mark.parametrize("cfg", [-1, 0, 2, 5, "simt"])
+def test_row_maxima_from_the_epilogue_feed_the_next_linears_quantizer(cfg):
+    """Two chained linears: the first also reports the largest magnitude it wrote per token, the second quantizes
+    that output in one pass with it. Every tensor against the oracle: the maxima equal the row absmax of the
+    first output, and the chain equals the two-pass path bit for bit."""
+    M, K1, N1, N2 = 300, 1024, 1552, 520
+    l1, l2 = synth.LinearSpec("chain1", M, K1, N1), synth.LinearSpec("chain2", M, N1, N2, bias=False)
+    t1, W2 = synth.make_linear(l1), synth.make_weight(l2)
+    t1["A"][5] = 0                                      # a zero token: its output row is the bias
+    qw1_ref, sch1_ref = oracle.quantize_weight_per_channel(t1["W"].numpy())
+    qw2_ref, sch2_ref = oracle.quantize_weight_per_channel(W2.numpy())
+    r1 = oracle.linear_fused_bf16(synth.bf16_bits(t1["A"]), qw1_ref, sch1_ref, t1["bias"].numpy())
+    rowmax_ref = oracle.row_absmax_bf16(r1["out"])
+    qa2_ref, stok2_ref = oracle.quantize_act_per_token_given_absmax(r1["out"], rowmax_ref)
+    r2 = oracle.linear_fused_int8(qa2_ref, stok2_ref, qw2_ref, sch2_ref, None)
+    assert np.array_equal(r2["out"], oracle.linear_fused_bf16(r1["out"], qw2_ref, sch2_ref, None)["out"])
+
+    qw1, sch1 = w8.int8_quantize_weight_per_channel(t1["W"].to(DEV))
+    qw2, sch2 = w8.int8_quantize_weight_per_channel(W2.to(DEV))
+    w8.force_config(n_tc_configs() if cfg == "simt" else cfg)
+    ws1 = w8.alloc_workspace(M, N1, K1, w8.ACT_BF16, DEV)
+    ws2 = w8.alloc_workspace(M, N2, N1, w8.ACT_BF16, DEV)
+    y1, rowmax = w8.int8_linear_fused_rowmax(t1["A"].to(DEV), qw1, sch1, t1["bias"].to(DEV), workspace=ws1)
+    y2, rowmax2 = w8.int8_linear_fused_rowmax(y1, qw2, sch2, None, workspace=ws2, rowmax_in=rowmax)
+    check_status(ws1)
+    check_status(ws2)
+    assert np.array_equal(synth.bf16_bits(y1.cpu()), r1["out"])
+    assert np.array_equal(rowmax.cpu().numpy().view(np.uint32), rowmax_ref.view(np.uint32))
+    s_off, q_off = w8.int8_linear_workspace_offsets(M, N1)
+    assert np.array_equal(ws2[q_off:q_off + M * N1].view(torch.int8).view(M, N1).cpu().numpy(), qa2_ref)
+    assert np.array_equal(ws2[s_off:s_off + 4 * M].view(torch.float32).cpu().numpy(), stok2_ref)
+    assert_bf16_close(synth.bf16_bits(y2.cpu()), r2["out"])
+    assert np.array_equal(rowmax2.cpu().numpy(), oracle.row_absmax_bf16(r2["out"]))
+    # input and output maxima must not share memory
+    lib = w8.binding.raw()
+    rc = lib.int8_linear_fused_given_absmax(y1.data_ptr(), N1, rowmax.data_ptr(), qw2.data_ptr(), sch2.data_ptr(), None,
+                                            y2.data_ptr(), N2, rowmax.data_ptr(), M, N2, N1, ws2.data_ptr(), ws2.numel(), None)
+    assert rc == 1
+
+
+def test_row_maxima_from_a_k_split_tile():
+    # the part that finishes a tile cut along K runs the epilogue from the summed slab: the maxima come from there too
+    spec = synth.LinearSpec("rowmax_split", 256, 8192, 264)
+    t = synth.make_linear(spec)
+    qw_ref, s_ch_ref = oracle.quantize_weight_per_channel(t["W"].numpy())
+    ref = oracle.linear_fused_bf16(synth.bf16_bits(t["A"]), qw_ref, s_ch_ref, t["bias"].numpy())
+    qw, s_ch = w8.int8_quantize_weight_per_channel(t["W"].to(DEV))
+    ws = w8.alloc_workspace(spec.M, spec.N, spec.K, w8.ACT_BF16, DEV)
+    assert w8.int8_linear_plan(spec.M, spec.N, spec.K, w8.ACT_BF16, ws.numel())["split_parts"] >= 2
+    y, rowmax = w8.int8_linear_fused_rowmax(t["A"].to(DEV), qw, s_ch, t["bias"].to(DEV), workspace=ws)
+    check_status(ws)
+    assert np.array_equal(synth.bf16_bits(y.cpu()), ref["out"])
+    assert np.array_equal(rowmax.cpu().numpy(), oracle.row_absmax_bf16(ref["out"]))
+
+
+# ------------------------------------------------------------------------------- wide items (two sub-tiles sharing A)
+
+WIDE_SHAPES = [
+    # (M, N, K, wide items per row block; None = the planner's choice)
+    (600, 1536, 512, None), (600, 1536, 512, 0), (600, 1536, 512, 1), (600, 1536, 512, 2), (600, 1536, 512, 3),
+    (300, 1288, 400, 2),      # ragged N: the last column block is partly outside, K tail inside a stage
+    (300, 1288, 400, 3),      # ... and inside the second half of a wide item
+    (130, 264, 160, 1),       # one wide item whose second half lies almost entirely outside N
+    (2816, 3072, 1024, 4),    # 11 row blocks x (4 wide + 4 narrow): every group gets several items of both kinds
+    (4608, 3072, 256, 6),     # all wide, 108 items on 74 groups
+]
+
+
+@pytest.mark.parametrize("M,N,K,w", WIDE_SHAPES)
+def test_wide_items_accumulators_and_outputs_bit_exact(M, N, K, w):
+    rng = np.random.default_rng(M + 7 * N + 11 * K + (0 if w is None else w))
+    qa, qw = rand_codes(rng, (M, K)), rand_codes(rng, (N, K))
+    s_tok = (rng.random(M) * 0.05 + 0.01).astype(np.float32)
+    s_ch = (rng.random(N) * 0.0008 + 0.0002).astype(np.float32)
+    bias = (rng.standard_normal(N) * 0.01).astype(np.float32)
+    ref = oracle.linear_fused_int8(qa, s_tok, qw, s_ch, bias)
+    dev = [torch.from_numpy(a).to(DEV) for a in (qa, qw, s_tok, s_ch, bias)]
+    wide_cfg = next(i for i in range(n_tc_configs()) if "2 x 256" in w8.config_name(i))
+    w8.force_config(wide_cfg if w is None else wide_cfg + ((w + 1) << 12))
+    ws = w8.alloc_workspace(M, N, K, w8.ACT_INT8, DEV)
+    assert w8.int8_linear_plan(M, N, K, w8.ACT_INT8, ws.numel())["config"] == wide_cfg
+    acc = w8.int8_gemm_i32_debug(dev[0], dev[1], ws)
+    check_status(ws)
+    assert np.array_equal(acc.cpu().numpy(), ref["acc"])
+    canvas = torch.full((M + 3, N + 24), -2.0, dtype=torch.bfloat16, device=DEV)     # guard band around the output
+    out = canvas[1:1 + M, 8:8 + N]
+    for _ in range(2):
+        w8.int8_linear_fused(dev[0], dev[1], dev[3], dev[4], s_tok=dev[2], out=out, workspace=ws)
+        check_status(ws)
+        assert_bf16_close(synth.bf16_bits(out.contiguous().cpu()), ref["out"])
+    mask = torch.ones_like(canvas, dtype=torch.bool)
+    mask[1:1 + M, 8:8 + N] = False
+    assert (canvas[mask] == -2.0).all()
+
+
 # ------------------------------------------------------------------------------- random shapes, every configuration
 
 def test_random_shapes_all_configurations_match_the_oracle():
