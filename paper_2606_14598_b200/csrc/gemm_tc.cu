@@ -649,8 +649,9 @@ constexpr TcConfig kConfigs[] = {
     // measured on the c4 shapes (hot L2): pair 256x256 3 x 256 B: 115 / 111 us; one CTA 128x256 4 x 128 B: 129 / 121 us;
     // pair 256x192: 130 / 123 us; one CTA 128x128: 164 / 154 us; pair 256x128: 168 / 162 us. Stage shapes of the
     // 256x256 pair at the same 192 KB: 6 x 128 B of K 126 / 118 us, 2 x 384 B 123 / 117 us (both directions lose).
-    // Pair tiles of two sub-tiles: 2 x 256 wins where K is deep and the wide items fill whole waves (M = 9472,
-    // K = 12288 -> N = 3072: 213-225 against 230-237 us); 2 x 192 lost everywhere (N = 192 MMAs) and is not built.
+    // Pair tiles of two sub-tiles: 2 x 256 wins cold bursts where K is deep and the wide items fill whole waves
+    // (M = 9472, K = 12288 -> N = 3072: 208-225 against 216-237 us) and loses once the power cap bites (see tc_plan);
+    // 2 x 192 lost everywhere (N = 192 MMAs) and is not built.
     {"tc 128x256 per CTA, 4 stages x 128 B of K", 1, 256, 1, 4, 1, 0.89f},
     {"tc 128x128 per CTA, 3 stages x 256 B of K", 1, 128, 1, 3, 2, 0.72f},
     {"tc 256x256 per CTA pair, 3 stages x 256 B of K", 2, 256, 1, 3, 2, 1.00f},
@@ -823,12 +824,15 @@ TcPlan tc_plan(int M, int N, int K, int forced, size_t scratch_bytes) {
         return plan_config(id, M, N, K, allow_split, false, scratch_bytes, wf, nullptr);   // forced: cut whenever possible
     }
     // lowest estimated time; on (near) ties the earlier entry of this preference order wins
-    constexpr int order[] = {2, 5, 0, 4, 3, 1};
+    // The configuration of two sub-tiles per tile is not among the candidates: alternating with the 256 x 256 pair in
+    // one process (M = 9216, K = 12288 -> N = 3072, 60 launches each) it won the first, cold round (208 against
+    // 216 us) and lost every later one (235-260 against 223-237 us): it keeps the tensor pipe busier, draws more
+    // power and is clocked down further (1.23-1.38 against 1.33-1.42 GHz measured inside the kernels). It stays
+    // available as a forced configuration.
+    constexpr int order[] = {2, 0, 4, 3, 1};
     TcPlan best{};
     double best_us = 0.0;
     for (int i = 0; i < static_cast<int>(sizeof(order) / sizeof(order[0])); ++i) {
-        // wide tiles expose one accumulator drain per item: measured to pay only where the k-loop is long
-        if (kConfigs[order[i]].nsub == 2 && K < 8192) continue;
         double us = 0.0;
         const TcPlan p = plan_config(order[i], M, N, K, allow_split, true, scratch_bytes, -1, &us);
         if (i == 0 || us < best_us * 0.97) { best = p; best_us = us; }

@@ -246,15 +246,18 @@ quant_rows_staged_kernel(const __nv_bfloat16* __restrict__ x, int64_t ld, int ro
         uint32_t phase = 0;
         bool ok = true;
         for (int g = blockIdx.x; g < total_groups; g += gridDim.x) {
+            const int row = g * RPS + slot;
+            // an absmax that is handed in is fetched while the row's bytes are still on their way (plain, coherent
+            // load: the value may have been written by the kernel ahead while this one was already resident)
+            float amax_given = 0.f;
+            if (GIVEN && row < rows) amax_given = __ldcg(amax_in + row);
             if (ok && !mbar_wait(full_bar(stage), phase, ctl, 2, kStatusTimeout)) ok = false;
             ok = __all_sync(0xffffffffu, ok) != 0;
-            const int row = g * RPS + slot;
             const bool live = ok && row < rows;
             const uint4* srow = reinterpret_cast<const uint4*>(base_ptr + stage * stage_bytes + slot * row_bytes);
             float amax = 0.f;
             if (GIVEN) {
-                // plain (coherent) load: the value may have been written by the kernel ahead while this one was resident
-                if (row < rows) amax = __ldcg(amax_in + row);
+                amax = amax_given;
             } else if (SMOOTH) {
                 if (live) {
 #pragma unroll 2
