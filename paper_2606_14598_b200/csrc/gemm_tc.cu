@@ -327,7 +327,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             auto release_stage = [&](int st) {
                 // (signalling only the leader and letting its producer pass the release on to the peer with a remote
                 // arrive was measured: 147 against 110 us on the MLP down-projection. The release -> refill latency
-                // is what this pipeline lives on.)
+                // is what this pipeline lives on. One commit with a CTA mask that arrives on both barriers at once
+                // measured the same as these two: 111.0 / 115.0 us.)
                 if (CG == 2) { tc_commit_pair(empty_bar(st)); tc_commit_pair(mapa_shared(empty_bar(st), 1)); }
                 else tc_commit(empty_bar(st));
             };
