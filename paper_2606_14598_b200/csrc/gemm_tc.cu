@@ -649,7 +649,8 @@ struct TcConfig {
 constexpr TcConfig kConfigs[] = {
     // measured on the c4 shapes (hot L2): pair 256x256 3 x 256 B: 115 / 111 us; one CTA 128x256 4 x 128 B: 129 / 121 us;
     // pair 256x192: 130 / 123 us; one CTA 128x128: 164 / 154 us; pair 256x128: 168 / 162 us. Stage shapes of the
-    // 256x256 pair at the same 192 KB: 6 x 128 B of K 126 / 118 us, 2 x 384 B 123 / 117 us (both directions lose).
+    // 256x256 pair at the same 192 KB: 6 x 128 B of K 126 / 118 us (120 / 114 us with a single commit per stage),
+    // 2 x 384 B 123 / 117 us (both directions lose).
     // Pair tiles of two sub-tiles: 2 x 256 wins cold bursts where K is deep and the wide items fill whole waves
     // (M = 9472, K = 12288 -> N = 3072: 208-225 against 216-237 us) and loses once the power cap bites (see tc_plan);
     // 2 x 192 lost everywhere (N = 192 MMAs) and is not built.
