@@ -86,16 +86,21 @@ __device__ __forceinline__ float unpack_max(__nv_bfloat162 m) {
 // instruction): the same sequence as quant1 on a pair of values held in one 64-bit register.
 struct RowScale2 {          // RowScale with its constants replicated into both halves
     uint64_t neg_s, inv, magic;
+    uint64_t inv_hi, inv_lo;        // the reciprocal in two pieces, for bf16 inputs (see quant2)
 };
 __device__ __forceinline__ RowScale2 make_row_scale2(const RowScale& rs) {
-    return RowScale2{pack2(-rs.s, -rs.s), pack2(rs.inv, rs.inv), pack2(MAGIC, MAGIC)};
+    // inv_hi: the reciprocal cut to 16 significant bits; inv_lo: what is missing to 1 / s, to ~2^-39 of it
+    const float inv_hi = __uint_as_float(__float_as_uint(rs.inv) & 0xffffff00u);
+    const float inv_lo = rs.fast ? __fdiv_rn(__fmaf_rn(-rs.s, inv_hi, 1.0f), rs.s) : 0.f;
+    return RowScale2{pack2(-rs.s, -rs.s), pack2(rs.inv, rs.inv), pack2(MAGIC, MAGIC), pack2(inv_hi, inv_hi), pack2(inv_lo, inv_lo)};
 }
-// codes of the two bf16 values of `w` in byte 0 and byte 4 of the result
+// Codes of the two bf16 values of `w` in byte 0 and byte 4 of the result. A bf16 value has 8 significant bits, so its
+// product with the 16-bit inv_hi is exact; one fma adds x * inv_lo and rounds once: a faithful quotient (within an ulp
+// of x / s) in two operations instead of three. The remainder pair then makes it the correctly rounded one as above.
 __device__ __forceinline__ uint64_t quant2(uint32_t w, const RowScale2& r2) {
     const uint64_t x = pack2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
-    const uint64_t q0 = mul2(x, r2.inv);
-    const uint64_t r0 = fma2(r2.neg_s, q0, x);
-    const uint64_t q1 = fma2(r0, r2.inv, q0);
+    const uint64_t p = mul2(x, r2.inv_hi);
+    const uint64_t q1 = fma2(x, r2.inv_lo, p);
     const uint64_t r1 = fma2(r2.neg_s, q1, x);
     const uint64_t q2 = fma2(r1, r2.inv, q1);
     return add2(q2, r2.magic);
