@@ -289,7 +289,9 @@ int int8_debug_set_starve(int mode);
  * but never cut tiles along K; id = that configuration; id + 0x100 = that configuration, never cut along K.
  * For the configuration whose tiles are two sub-tiles side by side, bits 12-19, if not zero, are 1 + the number of
  * such wide tiles per block of 256 rows (the remaining column blocks run as single sub-tiles); too large a
- * number falls back to the library's choice. Returns the previous value.
+ * number falls back to the library's choice. For the other tensor-core configurations bits 20-27, if not zero,
+ * are the height, in row blocks, of the bands the tiles are walked in (1 = along N first; by default the library
+ * bands the order only when the two int8 operands together exceed what stays in L2). Returns the previous value.
  */
 int int8_linear_force_config(int config_id);
 

@@ -118,7 +118,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                const __grid_constant__ CUtensorMap tm_out,
                const float* s_tok, const float* __restrict__ s_ch, const float* __restrict__ bias,
                int32_t* __restrict__ raw_out, int M, int N, int K, const RunCtl rc,
-               int split_tiles, int split_s, int32_t* split_slabs, int* split_counters, int wide_per_row,
+               int split_tiles, int split_s, int32_t* split_slabs, int* split_counters, int wide_per_row, int band,
                float* rowmax) {
     using L = SmemLayout<CG, BNS, NSUB, STAGES, KBS>;
     constexpr int BN = L::BN;
@@ -174,8 +174,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     constexpr int TILE_M = BM * CG;
     const int num_m = (M + TILE_M - 1) / TILE_M;
     const int num_nb = (N + BNS - 1) / BNS;                     // column blocks of one sub-tile's width
-    // Work items. NSUB = 1: one item per tile, along N first, then the next block of rows (banded orders were
-    // measured: no difference on the benchmark shapes, hot or cold L2). NSUB = 2: every block of rows is covered by
+    // Work items. NSUB = 1: one item per tile. With band = 1 they run along N first, then the next block of rows: a
+    // wave of concurrent tiles then shares a few row blocks of A and all of W, which is fine while both operands stay
+    // in L2. When they do not (the host decides), bands of `band` row blocks are walked column by column, so that a
+    // wave covers about as many row blocks as column blocks and fetches the fewest operand bytes from DRAM (its CTAs
+    // move along K in step, so within a wave every operand byte is fetched once). NSUB = 2: every block of rows is covered by
     // wide_per_row wide items (two column blocks side by side, sharing A) followed by narrow items (one column
     // block) for the rest; all wide items come first in the list, then all narrow ones, and item i belongs to CTA
     // group i mod groups. The host picks wide_per_row so that the groups end up with equal work (e.g. 18 x 12 column
@@ -197,8 +200,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     const int unit_sb = has_unit ? num_kstages * unit_part / split_s : 0;
     const int unit_se = has_unit ? num_kstages * (unit_part + 1) / split_s : 0;
     struct Item { int m0, n0, nsub; };                          // first row (of the pair), first column, sub-tiles
+    const int band_tiles = band * num_nb;                       // tiles of a full band (NSUB = 1)
     auto item = [&](int t) -> Item {
-        if (NSUB == 2 && t < num_wide) return Item{(t / wide_div) * TILE_M, (t % wide_div) * 2 * BNS, 2};
+        if (NSUB == 1) {
+            const int b = t / band_tiles, r = t - b * band_tiles;
+            const int rows_here = min(band, num_m - b * band);  // the last band may be lower
+            return Item{(b * band + r % rows_here) * TILE_M, (r / rows_here) * BNS, 1};
+        }
+        if (t < num_wide) return Item{(t / wide_div) * TILE_M, (t % wide_div) * 2 * BNS, 2};
         const int u = t - num_wide;
         return Item{(u / narrow_div) * TILE_M, (2 * wide + u % narrow_div) * BNS, 1};
     };
@@ -713,7 +722,8 @@ int launch_cfg(const GemmArgs& a, const TcPlan& plan, cudaStream_t st) {
                                        RAW ? static_cast<int32_t*>(a.out) : nullptr, a.M, a.N, a.K, rc,
                                        plan.split_tiles, plan.split_parts,
                                        reinterpret_cast<int32_t*>(static_cast<uint8_t*>(a.split_ws) + kCounterBytes),
-                                       static_cast<int*>(a.split_ws), plan.wide_per_row, a.raw_i32 ? nullptr : a.rowmax);
+                                       static_cast<int*>(a.split_ws), plan.wide_per_row, plan.band > 0 ? plan.band : 1,
+                                       a.raw_i32 ? nullptr : a.rowmax);
     return e == cudaSuccess ? W8A8_OK : W8A8_ERR_CUDA;
 }
 
@@ -739,10 +749,26 @@ int launch_by_id(const GemmArgs& a, const TcPlan& plan, cudaStream_t st) {
 // Configurations of two sub-tiles are never cut; their degree of freedom is how many of a row block's column
 // blocks are paired into wide items (see the kernel): the count that gives the busiest group the least work wins.
 TcPlan plan_config(int id, int M, int N, int K, bool allow_split, bool only_if_faster, size_t scratch_bytes, int wide_forced,
-                   double* est_us) {
+                   int band_forced, double* est_us) {
     const TcConfig& c = kConfigs[id];
     TcPlan p{};
     p.config = id;
+    p.band = 1;
+    if (c.nsub == 1) {
+        // Tile order: while both int8 operands stay in L2 (126 MB; 96 MB leaves room for the output on its way out)
+        // the tiles run along N first. Beyond that a wave of G concurrent tiles should span as many row blocks as
+        // column blocks: bands of about sqrt(G * BN / TILE_M) row blocks, walked column by column.
+        const int groups_all = sm_count() / c.cg;
+        const int rows_all = (M + BM * c.cg - 1) / (BM * c.cg);
+        if (band_forced > 0) {
+            p.band = band_forced;
+        } else if ((static_cast<double>(M) + N) * K > 96e6) {
+            int b = 1;
+            while ((b + 1) * (b + 1) * BM * c.cg <= groups_all * c.bns) ++b;
+            p.band = b;
+        }
+        if (p.band > rows_all) p.band = rows_all;
+    }
     const int max_groups = sm_count() / c.cg;
     const int num_m = (M + BM * c.cg - 1) / (BM * c.cg);
     const double fixed_us = 4.0;                       // launch, pipeline fill, last epilogue
@@ -816,14 +842,16 @@ const char* tc_config_name(int id) { return (id >= 0 && id < kNumConfigs) ? kCon
 
 TcPlan tc_plan(int M, int N, int K, int forced, size_t scratch_bytes) {
     // forced: -1 automatic, -2 automatic without K-split, id, or id + 0x100 for that configuration without K-split;
-    // bits 12-19, if not zero, are 1 + the number of wide items per row block (two-sub-tile configurations)
+    // bits 12-19, if not zero, are 1 + the number of wide items per row block (two-sub-tile configurations);
+    // bits 20-27, if not zero, are the band height in row blocks of the tile order (single-sub-tile configurations)
     const bool allow_split = forced == -1 || (forced >= 0 && (forced & kNoSplitBit) == 0);
     const int id = forced < 0 ? -1 : (forced & (kNoSplitBit - 1));
     const int wide_forced = forced < 0 ? -1 : ((forced >> 12) & 0xff) - 1;
+    const int band_forced = forced < 0 ? 0 : ((forced >> 20) & 0xff);          // 0 = from the sizes
     if (id >= 0 && id < kNumConfigs) {
         int wf = wide_forced;
         if (kConfigs[id].nsub == 2 && wf > ((N + kConfigs[id].bns - 1) / kConfigs[id].bns) / 2) wf = -1;   // not possible: choose
-        return plan_config(id, M, N, K, allow_split, false, scratch_bytes, wf, nullptr);   // forced: cut whenever possible
+        return plan_config(id, M, N, K, allow_split, false, scratch_bytes, wf, band_forced, nullptr);   // forced: cut whenever possible
     }
     // lowest estimated time; on (near) ties the earlier entry of this preference order wins
     // The configuration of two sub-tiles per tile is not among the candidates: alternating with the 256 x 256 pair in
@@ -836,7 +864,7 @@ TcPlan tc_plan(int M, int N, int K, int forced, size_t scratch_bytes) {
     double best_us = 0.0;
     for (int i = 0; i < static_cast<int>(sizeof(order) / sizeof(order[0])); ++i) {
         double us = 0.0;
-        const TcPlan p = plan_config(order[i], M, N, K, allow_split, true, scratch_bytes, -1, &us);
+        const TcPlan p = plan_config(order[i], M, N, K, allow_split, true, scratch_bytes, -1, 0, &us);
         if (i == 0 || us < best_us * 0.97) { best = p; best_us = us; }
     }
     return best;

@@ -102,9 +102,11 @@ struct TcPlan {
     int split_parts;       // parts per such tile
     size_t scratch_bytes;  // scratch the split needs (counters, then one int32 slab per tile); all zero at launch
     int wide_per_row;      // configurations of two sub-tiles: wide items (two column blocks) per block of rows
+    int band;              // other configurations: row blocks per band of the tile order (1 = along N first)
 };
 // Picks a configuration for the shape (or `forced` if >= 0; forced + 0x100 = that configuration without K-split;
-// bits 12-19 of `forced`, if not zero, are 1 + the number of wide items per block of rows).
+// bits 12-19 of `forced`, if not zero, are 1 + the number of wide items per block of rows; bits 20-27, if not zero,
+// the band height of the tile order).
 // A split is planned only if its scratch fits in scratch_bytes.
 TcPlan tc_plan(int M, int N, int K, int forced, size_t scratch_bytes);
 // Scratch the automatic choice uses when it is given enough.

@@ -590,6 +590,31 @@ def test_wide_items_accumulators_and_outputs_bit_exact(M, N, K, w):
     assert (canvas[mask] == -2.0).all()
 
 
+# ------------------------------------------------------------------------------- banded tile order
+
+@pytest.mark.parametrize("M,N,K,cfg,band", [(1300, 1288, 400, 2, 2), (1300, 1288, 400, 2, 3), (1300, 1288, 400, 2, 8),
+                                             (700, 2056, 272, 0, 4), (520, 1032, 4096, 2, 2), (300, 520, 2064, 4, 5)])
+def test_banded_tile_order_is_bit_exact(M, N, K, cfg, band):
+    # bands of row blocks walked column by column (the order used when the operands exceed L2), forced on small
+    # shapes: ragged last band, ragged edges, and a shape whose partial wave is cut along K
+    rng = np.random.default_rng(M + 3 * N + 5 * K + band)
+    qa, qw = rand_codes(rng, (M, K)), rand_codes(rng, (N, K))
+    s_tok = (rng.random(M) * 0.05 + 0.01).astype(np.float32)
+    s_ch = (rng.random(N) * 0.0008 + 0.0002).astype(np.float32)
+    bias = (rng.standard_normal(N) * 0.01).astype(np.float32)
+    ref = oracle.linear_fused_int8(qa, s_tok, qw, s_ch, bias)
+    dev = [torch.from_numpy(a).to(DEV) for a in (qa, qw, s_tok, s_ch, bias)]
+    w8.force_config(cfg + (band << 20))
+    ws = w8.alloc_workspace(M, N, K, w8.ACT_INT8, DEV)
+    ws = torch.empty(ws.numel() + (16 << 20), dtype=torch.uint8, device=DEV)
+    acc = w8.int8_gemm_i32_debug(dev[0], dev[1], ws)
+    check_status(ws)
+    assert np.array_equal(acc.cpu().numpy(), ref["acc"])
+    out = w8.int8_linear_fused(dev[0], dev[1], dev[3], dev[4], s_tok=dev[2], workspace=ws)
+    check_status(ws)
+    assert_bf16_close(synth.bf16_bits(out.cpu()), ref["out"])
+
+
 # ------------------------------------------------------------------------------- random shapes, every configuration
 
 def test_random_shapes_all_configurations_match_the_oracle():
