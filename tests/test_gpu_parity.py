@@ -336,17 +336,26 @@ def test_fused_from_bf16_with_row_stride_no_bias_and_k_split():
     assert (wide[:, :8] == 7.0).all() and (wide[:, 8 + spec.K:] == 7.0).all()
 
 
-@pytest.mark.parametrize("M", [1, 2, 5, 16])
-def test_skinny_m_path(M):
-    spec = synth.LinearSpec(f"skinny{M}", M, 3072, 2048, outlier_frac=0.0)
+@pytest.mark.parametrize("M,K,N", [(1, 3072, 2048), (2, 3072, 2048), (5, 3072, 2048), (16, 3072, 2048),
+                                   (3, 3072, 2056), (4, 1024, 4104), (2, 6144, 1032), (2, 16, 1024), (2, 12288, 1544),
+                                   (2, 3072, 18432)])
+def test_skinny_m_path(M, K, N):
+    # M <= 4 with enough weight rows: the weight-streaming kernel (ring of bulk copies); M = 5 and rows too long for a
+    # three-stage ring: the register kernel; M = 16: the tensor-core path
+    spec = synth.LinearSpec(f"skinny{M}x{K}x{N}", M, K, N, outlier_frac=0.0)
     t = synth.make_linear(spec)
     qw_ref, s_ch_ref = oracle.quantize_weight_per_channel(t["W"].numpy())
     ref = oracle.linear_fused_bf16(synth.bf16_bits(t["A"]), qw_ref, s_ch_ref, t["bias"].numpy())
     qw, s_ch = w8.int8_quantize_weight_per_channel(t["W"].to(DEV))
     ws = w8.alloc_workspace(M, spec.N, spec.K, w8.ACT_BF16, DEV)
-    out = w8.int8_linear_fused(t["A"].to(DEV), qw, s_ch, t["bias"].to(DEV), workspace=ws)
+    out, rowmax = w8.int8_linear_fused_rowmax(t["A"].to(DEV), qw, s_ch, t["bias"].to(DEV), workspace=ws)
     check_status(ws)
     assert_bf16_close(synth.bf16_bits(out.cpu()), ref["out"])
+    assert np.array_equal(rowmax.cpu().numpy(), oracle.row_absmax_bf16(ref["out"]))
+    s_off, q_off = w8.int8_linear_workspace_offsets(M, K)
+    qa = ws[q_off:q_off + M * K].view(torch.int8).view(M, K)
+    acc = w8.int8_gemm_i32_debug(qa, qw)
+    assert np.array_equal(acc.cpu().numpy(), ref["acc"])
 
 
 def test_run_to_run_identical_and_host_buffer_entry_point():
