@@ -26,6 +26,9 @@
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
  *     Calls only enqueue work on it and return; they do not synchronize unless
  *     stated.
+ *   - The first call of a compute entry point on a device does one-time set-up for that device (function
+ *     attributes, the address of the library's sticky status word); make it outside any stream capture. Later
+ *     calls only enqueue kernel launches and at most two memsets and can be captured in a CUDA graph.
  *   - The return value is a w8a8_status. Argument errors are detected before
  *     anything is enqueued. There is no CPU fallback and no other backend: on a
  *     device that is not sm_100 (compute capability 10.0) the compute calls return W8A8_ERR_ARCH.

@@ -770,6 +770,47 @@ def test_benchmark_configs_full_size(spec):
     assert torch.equal(out2, out)
 
 
+# ------------------------------------------------------------------------------- more than 2^31 elements
+
+def test_quantizer_beyond_two_to_the_31_elements():
+    # 41 repeats of a 1000-row block of 104 KB rows: 2.18e9 activations. Every repeat must carry the codes the oracle
+    # gives for the block (an index that wrapped at 2^31 would read or write the wrong rows).
+    K, rows, reps = 53248, 1000, 41
+    assert rows * reps * K > 2 ** 31
+    block = synth.make_activations(synth.LinearSpec("big_q", rows, K, 8))
+    qa_ref, s_ref = oracle.quantize_act_per_token(synth.bf16_bits(block))
+    A = block.to(DEV).repeat(reps, 1)
+    qa, s = w8.int8_quantize_act_per_token(A)
+    del A
+    qa_ref_d, s_ref_d = torch.from_numpy(qa_ref).to(DEV), torch.from_numpy(s_ref).to(DEV)
+    assert torch.equal(s.view(reps, rows), s_ref_d.expand(reps, rows))
+    for r in range(reps):
+        assert torch.equal(qa[r * rows:(r + 1) * rows], qa_ref_d), r
+
+
+def test_fused_output_beyond_two_to_the_31_elements():
+    # 46400 x 46400 outputs (2.15e9, 4.3 GB of bf16) from a short K: the activation rows repeat a 928-row block, so
+    # every block of output rows must equal the oracle's result for that block.
+    M, N, K, rows = 46400, 46400, 64, 928
+    assert M * N > 2 ** 31 and M % rows == 0
+    rng = np.random.default_rng(31)
+    qa_b, qw = rand_codes(rng, (rows, K)), rand_codes(rng, (N, K))
+    s_tok_b = (rng.random(rows) * 0.05 + 0.01).astype(np.float32)
+    s_ch = (rng.random(N) * 0.0008 + 0.0002).astype(np.float32)
+    bias = (rng.standard_normal(N) * 0.01).astype(np.float32)
+    ref = torch.from_numpy(oracle.linear_fused_int8(qa_b, s_tok_b, qw, s_ch, bias)["out"].view(np.int16)).to(DEV)
+    reps = M // rows
+    qa = torch.from_numpy(qa_b).to(DEV).repeat(reps, 1)
+    s_tok = torch.from_numpy(s_tok_b).to(DEV).repeat(reps)
+    ws = w8.alloc_workspace(M, N, K, w8.ACT_INT8, DEV)
+    out = w8.int8_linear_fused(qa, torch.from_numpy(qw).to(DEV), torch.from_numpy(s_ch).to(DEV), torch.from_numpy(bias).to(DEV),
+                               s_tok=s_tok, workspace=ws)
+    check_status(ws)
+    got = out.view(torch.int16)
+    for r in range(reps):
+        assert torch.equal(got[r * rows:(r + 1) * rows], ref), r
+
+
 # ------------------------------------------------------------------------------- bounded waits that run out
 
 @pytest.fixture
