@@ -18,7 +18,6 @@ import json
 import os
 import statistics
 import sys
-import threading
 import time
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
@@ -54,62 +53,88 @@ def measured_peaks():
 
 # ------------------------------------------------------------------------------------------ clocks
 
+SAMPLER_SRC = r"""
+import json, sys, time
+idx, period = sys.argv[1], float(sys.argv[2])
+import pynvml as nv
+nv.nvmlInit()
+h = nv.nvmlDeviceGetHandleByIndex(int(idx)) if idx.isdigit() else nv.nvmlDeviceGetHandleByUUID(idx)
+print(json.dumps({"max_mhz": float(nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM))}), flush=True)
+while True:
+    t = time.time()
+    try:
+        mhz = float(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
+        pw = nv.nvmlDeviceGetPowerUsage(h) / 1000.0
+        try:
+            mask = nv.nvmlDeviceGetCurrentClocksEventReasons(h)
+        except Exception:
+            mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+        sys.stdout.write(json.dumps({"t": t, "mhz": mhz, "w": pw, "mask": int(mask)}) + "\n")
+        sys.stdout.flush()
+    except Exception:
+        pass
+    time.sleep(period)
+"""
+
+
 class ClockSampler:
-    """Samples SM clock, power and clock-event reasons through NVML while the timed region runs."""
+    """Samples SM clock, power and clock-event reasons through NVML while the timed region runs. The sampling loop is
+    a process of its own (a thread of this one is starved by the launch loop), started ahead of the warm-up; only the
+    samples whose time stamps fall between enter and exit are kept."""
 
     REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap",
                0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting", 0x100: "display_clock_setting",
                0x10: "sync_boost"}
 
     def __init__(self, index: int, period_s: float = 0.002):
-        self.period = period_s
+        import subprocess
         self.samples, self.power, self.reasons = [], [], set()
-        self.max_mhz = None
-        self._stop = threading.Event()
-        self._thr = None
+        self.max_mhz, self.t0, self.t1, self.proc = None, None, None, None
+        visible = os.environ.get("CUDA_VISIBLE_DEVICES")
+        tok = str(index)
+        if visible:
+            ids = [v for v in visible.split(",") if v.strip() != ""]
+            tok = ids[index] if index < len(ids) else ids[0]
         try:
-            import pynvml
-            pynvml.nvmlInit()
-            self.nv = pynvml
-            visible = os.environ.get("CUDA_VISIBLE_DEVICES")
-            if visible:
-                ids = [v for v in visible.split(",") if v.strip() != ""]
-                tok = ids[index] if index < len(ids) else ids[0]
-                self.h = pynvml.nvmlDeviceGetHandleByIndex(int(tok)) if tok.isdigit() else pynvml.nvmlDeviceGetHandleByUUID(tok)
-            else:
-                self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
-            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.proc = subprocess.Popen([sys.executable, "-c", SAMPLER_SRC, tok, str(period_s)], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            first = self.proc.stdout.readline()            # the sampler is up once it has printed the maximum clock
+            self.max_mhz = json.loads(first)["max_mhz"] if first else None
+            if self.max_mhz is None:
+                raise RuntimeError("no answer from the sampler")
         except Exception as e:          # NVML missing: report that no clocks were sampled
-            log(f"[bench] NVML unavailable: {e}")
-            self.nv = None
+            log(f"[bench] NVML sampler unavailable: {e}")
+            self.close()
 
-    def _loop(self):
-        nv = self.nv
-        while not self._stop.is_set():
-            try:
-                self.samples.append(float(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
-                self.power.append(nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0)
-                try:
-                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
-                except Exception:
-                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
-                for bit, name in self.REASONS.items():
-                    if mask & bit:
-                        self.reasons.add(name)
-            except Exception:
-                pass
-            self._stop.wait(self.period)
+    def close(self):
+        if self.proc is not None:
+            self.proc.kill()
+            self.proc.wait()
+            self.proc = None
 
     def __enter__(self):
-        if self.nv is not None:
-            self._thr = threading.Thread(target=self._loop, daemon=True)
-            self._thr.start()
+        self.t0 = time.time()
         return self
 
     def __exit__(self, *exc):
-        self._stop.set()
-        if self._thr is not None:
-            self._thr.join()
+        self.t1 = time.time()
+        if self.proc is None:
+            return
+        time.sleep(0.01)
+        self.proc.kill()
+        out, _ = self.proc.communicate()
+        self.proc = None
+        for ln in out.splitlines():
+            try:
+                d = json.loads(ln)
+            except Exception:
+                continue
+            if "t" in d and self.t0 <= d["t"] <= self.t1:
+                self.samples.append(d["mhz"])
+                self.power.append(d["w"])
+                for bit, name in self.REASONS.items():
+                    if d["mask"] & bit:
+                        self.reasons.add(name)
 
     def summary(self):
         if not self.samples:
@@ -224,7 +249,7 @@ def main():
                     help="graph: each step is one replay of a captured CUDA graph of the step's calls; direct: the calls themselves")
     ap.add_argument("--config", type=int, default=-1, help="force a kernel configuration (sweeps); -1 = from the shape")
     ap.add_argument("--repeats", type=int, default=0,
-                    help="timed loops of --steps steps (0 = 5, more for short loops so that clocks get sampled); the median is reported")
+                    help="timed loops of --steps steps (0 = 7, enough for ten NVML samples over 20-step loops); the median is reported")
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         # no launcher: run one process per GPU ourselves (rank i on GPU i); the ranks meet through a rendezvous file
@@ -305,6 +330,7 @@ def main():
         del a, b
 
     # ---- the timed region
+    clocks = ClockSampler(local_rank)                      # its process starts now and samples through the warm-up too
     for i in range(max(args.warmup, len(step_args))):      # direct calls first: one-time set-up happens outside any capture
         step(i)
     torch.cuda.synchronize()
@@ -353,9 +379,9 @@ def main():
     # R timed loops of exactly --steps steps each, every one bracketed by a barrier and a device synchronize on both
     # sides and timed with CUDA events on the launching stream; a loop's time is the maximum over the ranks, the
     # reported value is the median loop. NVML is sampled every 2 ms across all of them.
-    repeats = args.repeats if args.repeats > 0 else 5
+    repeats = args.repeats if args.repeats > 0 else 7
     loop_sec = []
-    with ClockSampler(local_rank) as clocks:
+    with clocks:
         for _ in range(repeats):
             wdist.barrier(dev)
             torch.cuda.synchronize()
