@@ -433,7 +433,7 @@ def main():
                    "l2": f"inputs larger than L2: {len(sets)} rotating sets of {set_bytes / 1e6:.0f} MB each",
                    "parallelism": f"dp{world} over tokens, weights replicated, no collective"},
         "pct_of_int8_peak": 100.0 * tops / (INT8_PEAK_TOPS * world), "int8_peak_tops": INT8_PEAK_TOPS,
-        "clocks": clocks.summary(), "gpu_launches": launches,
+        "clocks": clocks.summary(), "gpu_launches": launches, "gpu_launches_all_loops": launches * repeats,
         "repeats": {"loops": repeats, "ms_per_step": [t / args.steps * 1e3 for t in loop_sec],
                     "tops": [ops_all_ranks / t / 1e12 for t in loop_sec], "reported": "median"},
     }
