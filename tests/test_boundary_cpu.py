@@ -60,12 +60,13 @@ def test_workspace_sizes():
 
 def test_plan_of_the_benchmark_shapes():
     # the static per-shape choice (148 SMs assumed without a device): CTA pairs with 256x256 tiles on the large
-    # shapes; deep K with a nearly empty last wave is cut along K when the workspace has room, and only then
+    # shapes; deep K with a nearly empty last wave is cut along K when the workspace has room, and only then.
+    # From three waves of tiles on, the grid is the fewest pairs that need no more waves (216 tiles: 72 pairs x 3).
     w8.force_config(-1)
     pair = next(i for i in range(w8.num_configs()) if "256x256 per CTA pair" in w8.config_name(i))
-    for (M, N, K) in [(4608, 12288, 3072), (4608, 3072, 12288), (9216, 9216, 3072), (2816, 3072, 3072)]:
+    for (M, N, K, groups) in [(4608, 12288, 3072, 72), (4608, 3072, 12288, 72), (9216, 9216, 3072, 72), (2816, 3072, 3072, 74)]:
         p = w8.int8_linear_plan(M, N, K, w8.ACT_BF16)
-        assert p["config"] == pair and p["split_parts"] == 0 and p["groups"] == 74, p
+        assert p["config"] == pair and p["split_parts"] == 0 and p["groups"] == groups, p
     p = w8.int8_linear_plan(4110, 4608, 53248, w8.ACT_BF16)
     assert p["config"] == pair and p["groups"] == 74 and p["split_tiles"] == 306 % 74 and p["split_parts"] == 7, p
     lo = w8.int8_linear_workspace_min_bytes(4110, 4608, 53248, w8.ACT_BF16)
