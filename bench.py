@@ -131,7 +131,8 @@ class ClockSampler:
                 continue
             if "t" in d and self.t0 <= d["t"] <= self.t1:
                 self.samples.append(d["mhz"])
-                self.power.append(d["w"])
+                if d["w"] is not None:
+                    self.power.append(d["w"])
                 for bit, name in self.REASONS.items():
                     if d["mask"] & bit:
                         self.reasons.add(name)
