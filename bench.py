@@ -381,6 +381,16 @@ def main():
     # sides and timed with CUDA events on the launching stream; a loop's time is the maximum over the ranks, the
     # reported value is the median loop. NVML is sampled every 2 ms across all of them.
     repeats = args.repeats if args.repeats > 0 else 7
+    if args.repeats <= 0:
+        # short loops (small workloads): more of them, so that the loops together last ~40 ms and NVML gets its samples
+        t0_, t1_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0_.record()
+        for i in range(args.steps):
+            run_step(i)
+        t1_.record()
+        torch.cuda.synchronize()
+        est = max(t0_.elapsed_time(t1_) * 1e-3, 1e-6)
+        repeats = int(wdist.max_over_ranks(float(max(7, min(200, int(0.04 / est) + 1))), dev))
     loop_sec = []
     with clocks:
         for _ in range(repeats):
