@@ -9,6 +9,7 @@
 
 #include <cuda_runtime.h>
 
+#include <cmath>
 #include <cstdint>
 #include <cstdio>
 #include <cstring>
@@ -19,6 +20,12 @@ static uint16_t f2bf(float f) {            // round to nearest even
     std::memcpy(&u, &f, 4);
     u += 0x7fffu + ((u >> 16) & 1u);
     return static_cast<uint16_t>(u >> 16);
+}
+static float bf2f(uint16_t h) {
+    uint32_t u = static_cast<uint32_t>(h) << 16;
+    float f;
+    std::memcpy(&f, &u, 4);
+    return f;
 }
 
 #define CK(x) do { if ((x) != cudaSuccess) { std::printf("CUDA error at line %d\n", __LINE__); return 2; } } while (0)
@@ -69,6 +76,32 @@ int main() {
             t = t + bias[n];
             if (out[m * N + n] != f2bf(t)) ++bad;
         }
+    // The same linear once more through the entry that also reports the largest magnitude written per token, then
+    // the one-pass quantizer on that output with those maxima: scales are rowmax / 127 (one float division) and the
+    // codes rne(x / s), both recomputed here in plain float arithmetic from the values worked out above.
+    float *drowmax, *ds2;
+    int8_t* dq2;
+    CK(cudaMalloc(&drowmax, M * 4)); CK(cudaMalloc(&ds2, M * 4)); CK(cudaMalloc(&dq2, M * N));
+    W8(int8_linear_fused_rowmax(dA, W8A8_ACT_BF16, K, nullptr, dqw, ds_ch, dbias, dout, N, drowmax, M, N, K, dws, ws_bytes, st));
+    W8(int8_check_status(dws, st));
+    W8(int8_quantize_act_per_token_given_absmax(dout, M, N, N, drowmax, dq2, ds2, st));
+    W8(int8_sticky_status(1, st));
+    std::vector<float> rowmax(M), s2(M);
+    std::vector<int8_t> q2(M * N);
+    CK(cudaMemcpy(rowmax.data(), drowmax, M * 4, cudaMemcpyDeviceToHost));
+    CK(cudaMemcpy(s2.data(), ds2, M * 4, cudaMemcpyDeviceToHost));
+    CK(cudaMemcpy(q2.data(), dq2, q2.size(), cudaMemcpyDeviceToHost));
+    for (int64_t m = 0; m < M; ++m) {
+        float want_max = 0.f;
+        for (int64_t n = 0; n < N; ++n) want_max = std::fmax(want_max, std::fabs(bf2f(out[m * N + n])));
+        const float want_s = want_max > 0.f ? want_max / 127.0f : 1.0f;
+        if (rowmax[m] != want_max || s2[m] != want_s) { ++bad; continue; }
+        for (int64_t n = 0; n < N; ++n) {
+            const volatile float quot = bf2f(out[m * N + n]) / want_s;      // volatile: one rounded float division
+            if (q2[m * N + n] != static_cast<int8_t>(std::nearbyintf(quot))) ++bad;   // default rounding mode: ties to even
+        }
+    }
+    cudaFree(drowmax); cudaFree(ds2); cudaFree(dq2);
     std::printf(bad == 0 ? "c client ok: %ld x %ld x %ld through the C ABI, every output as worked out by hand\n"
                          : "c client FAILED (%ld x %ld x %ld)\n", static_cast<long>(M), static_cast<long>(K), static_cast<long>(N));
     if (bad) std::printf("%ld mismatches\n", bad);
