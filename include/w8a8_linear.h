@@ -26,6 +26,12 @@
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
  *     Calls only enqueue work on it and return; they do not synchronize unless
  *     stated.
+ *   - Calls are chained on the stream with programmatic dependent launch: a kernel may be set up, and the GEMM may
+ *     already request its first WEIGHT tiles, while the kernel ahead of it on the stream is still finishing; it
+ *     waits for that kernel before it reads activations, their scales, per-channel scales or bias, and before it
+ *     writes anything. Weights (qw) must therefore be complete before the call is enqueued, or be written by
+ *     int8_quantize_weight_per_channel (which does not release its dependents early), by a copy, or by a kernel
+ *     that does not use cudaTriggerProgrammaticLaunchCompletion / griddepcontrol.launch_dependents.
  *   - The first call of a compute entry point on a device does one-time set-up for that device (function
  *     attributes, the address of the library's sticky status word); make it outside any stream capture. Later
  *     calls only enqueue kernel launches and at most two memsets and can be captured in a CUDA graph.

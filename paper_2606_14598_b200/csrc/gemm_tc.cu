@@ -217,7 +217,57 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         // ------------------------------------------------------------ TMA producer (both CTAs of a pair)
         // The kernel is always launched so that it may start while the kernel ahead of it in the stream is finishing
         // (the quantizer, or whatever the caller ran): everything up to here touched no global memory.
+        int stage = 0;
+        uint32_t phase = 0;
+        int issued = 0;
+        bool ok = true;
+        bool withhold = rc.starve != 0;                     // test hook: this CTA's very first stage never arrives
+        const uint64_t keep = l2_policy_evict_last();       // operands are re-read by other tiles: keep them in L2
+        // the loads of pipeline stage `ks` of item `it` into ring slot `st`: the barrier's byte count (armed once per
+        // k-block), the A tile and / or the W tile(s). A stage always receives all its k-blocks: those past the end of
+        // K are zero-filled by TMA (and skipped by the MMA thread), which keeps the byte count of the barrier constant.
+        auto load_stage = [&](const Item& it, int ks, int st, bool arm, bool load_a, bool load_b) {
+            const int m0 = it.m0 + rank * BM;
+            const int n0 = it.n0 + rank * L::B_ROWS;
+            const uint32_t kb_bytes = L::A_BYTES + it.nsub * L::B_BYTES;
+#pragma unroll
+            for (int sub = 0; sub < KBS; ++sub) {
+                const uint32_t sa = base + st * L::STAGE_BYTES + sub * L::KB_BYTES;
+                const int kx = (ks * KBS + sub) * BK;
+                if (CG == 2) {
+                    // the leader's barrier counts the bytes of both CTAs
+                    if (arm && leader) mbar_arrive_expect_tx(full_bar(st, sub), 2 * kb_bytes);
+                    const uint32_t fb = mapa_shared(full_bar(st, sub), 0);
+                    if (load_a) tma_load_2d_pair_hint(sa, &tm_a, fb, kx, m0, keep);
+#pragma unroll
+                    for (int h = 0; h < NSUB; ++h)
+                        if (load_b && h < it.nsub) tma_load_2d_pair_hint(sa + L::A_BYTES + h * L::B_BYTES, &tm_b, fb, kx, n0 + h * BNS, keep);
+                } else {
+                    if (arm) mbar_arrive_expect_tx(full_bar(st, sub), kb_bytes);
+                    if (load_a) tma_load_2d_hint(sa, &tm_a, full_bar(st, sub), kx, m0, keep);
+#pragma unroll
+                    for (int h = 0; h < NSUB; ++h)
+                        if (load_b && h < it.nsub) tma_load_2d_hint(sa + L::A_BYTES + h * L::B_BYTES, &tm_b, full_bar(st, sub), kx, n0 + h * BNS, keep);
+                }
+            }
+        };
+        // The first piece of work of this CTA group (a whole item, or its part of a tile cut along K).
+        const bool first_is_unit = !(first_tile < tiles_whole);
+        const int first_t = first_is_unit ? unit_tile : first_tile;
+        const int first_sb = first_is_unit ? unit_sb : 0, first_se = first_is_unit ? unit_se : num_kstages;
+        const bool any_work = first_tile < tiles_whole || has_unit;
+        int pre = 0;                                        // stages of that piece whose W tiles were requested early
         if (lane == 0) {
+            // The weights do not depend on the kernel ahead of this one (the quantizer writes activations): the W tiles
+            // of the first ring of stages are requested before the wait, the A tiles after it, so that the first MMA
+            // waits for the short trip of the freshly written activations out of L2 rather than for cold weights out
+            // of DRAM. (Weights, like every operand but the activations and their scales, must therefore be complete
+            // before the call is enqueued, or be written by a kernel that does not release its dependents early.)
+            if (any_work && !withhold) {
+                const Item it = item(first_t);
+                pre = min(STAGES, first_se - first_sb);
+                for (int i = 0; i < pre; ++i) load_stage(it, first_sb + i, i, true, false, true);   // the ring starts empty
+            }
             grid_dep_wait();
             // without a quantizer ahead of it (which clears the status word) the kernel clears it itself; a time-out
             // can only be recorded a whole wait limit later
@@ -229,23 +279,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 stamps[0] = static_cast<unsigned long long>(clock64());
                 stamps[1] = globaltimer_ns();
             }
+            if (pre > 0) {
+                const Item it = item(first_t);
+                for (int i = 0; i < pre; ++i) load_stage(it, first_sb + i, i, false, true, false);
+                issued = pre;
+                stage = pre == STAGES ? 0 : pre;
+                phase = pre == STAGES ? 1u : 0u;
+            }
         }
         __syncwarp();
-        int stage = 0;
-        uint32_t phase = 0;
-        int issued = 0;
-        bool ok = true;
-        bool withhold = rc.starve != 0;                     // test hook: this CTA's very first stage never arrives
-        auto produce = [&](int t, int sb, int se) {
+        // stages [sb, se) of item t; the first `skip` of them have been issued already
+        auto produce = [&](int t, int sb, int se, int skip) {
             const Item it = item(t);
-            const int m0 = it.m0 + rank * BM;
-            const int n0 = it.n0 + rank * L::B_ROWS;
-            const int nsub = it.nsub;
-            const uint32_t kb_bytes = L::A_BYTES + nsub * L::B_BYTES;
             if (lane == 0) {
-                const uint64_t keep = l2_policy_evict_last();        // operands are re-read by other tiles: keep them in L2
-                for (int ks = sb; ks < se; ++ks) {
-                    const int kb = ks * KBS;
+                for (int ks = sb + skip; ks < se; ++ks) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, ctl, W_PRODUCER_EMPTY, kStatusTimeout)) { ok = false; break; }
                     if (withhold) {
                         // neither the byte count nor a copy is posted for this stage: its barriers never complete, the
@@ -254,36 +301,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                         if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                         continue;
                     }
-                    // a stage always receives all its k-blocks: those past the end of K are zero-filled by TMA
-                    // (and skipped by the MMA thread), which keeps the byte count of the barrier constant
-#pragma unroll
-                    for (int sub = 0; sub < KBS; ++sub) {
-                        const uint32_t sa = base + stage * L::STAGE_BYTES + sub * L::KB_BYTES;
-                        const int kx = (kb + sub) * BK;
-                        if (CG == 2) {
-                            // the leader's barrier counts the bytes of both CTAs
-                            if (leader) mbar_arrive_expect_tx(full_bar(stage, sub), 2 * kb_bytes);
-                            const uint32_t fb = mapa_shared(full_bar(stage, sub), 0);
-                            tma_load_2d_pair_hint(sa, &tm_a, fb, kx, m0, keep);
-#pragma unroll
-                            for (int h = 0; h < NSUB; ++h)
-                                if (h < nsub) tma_load_2d_pair_hint(sa + L::A_BYTES + h * L::B_BYTES, &tm_b, fb, kx, n0 + h * BNS, keep);
-                        } else {
-                            mbar_arrive_expect_tx(full_bar(stage, sub), kb_bytes);
-                            tma_load_2d_hint(sa, &tm_a, full_bar(stage, sub), kx, m0, keep);
-#pragma unroll
-                            for (int h = 0; h < NSUB; ++h)
-                                if (h < nsub) tma_load_2d_hint(sa + L::A_BYTES + h * L::B_BYTES, &tm_b, full_bar(stage, sub), kx, n0 + h * BNS, keep);
-                        }
-                    }
+                    load_stage(it, ks, stage, true, true, true);
                     ++issued;
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
             ok = __all_sync(0xffffffffu, ok) != 0;
         };
-        for (int t = first_tile; t < tiles_whole && ok; t += tile_step) produce(t, 0, num_kstages);
-        if (has_unit && ok) produce(unit_tile, unit_sb, unit_se);
+        for (int t = first_tile; t < tiles_whole && ok; t += tile_step) produce(t, 0, num_kstages, t == first_t ? pre : 0);
+        if (has_unit && ok) produce(unit_tile, unit_sb, unit_se, first_is_unit ? pre : 0);
         if (!ok && lane == 0 && (CG == 1 || leader)) {
             // let copies that are still in flight land before the CTA goes away
             int s = stage;

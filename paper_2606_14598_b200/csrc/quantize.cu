@@ -396,7 +396,10 @@ quant_rows_kernel(const T* __restrict__ x, int64_t ld, int rows, int K,
         c.load(row + chunk * 16);
         if constexpr (SMOOTH) c.scale(mult + chunk * 16);
     };
-    grid_dep_launch_dependents();
+    // Activations: a dependent kernel (the GEMM) may set itself up while this one runs; it waits for this grid before it
+    // reads them. Weights (fp32 input) are different: the GEMM requests its first weight tiles before that wait, so the
+    // kernel that writes them must not release its dependents before it is complete.
+    if (!std::is_same<T, float>::value) grid_dep_launch_dependents();
     grid_dep_wait();                      // launched early behind a kernel that allowed it: wait for that kernel's results
     if (status != nullptr && blockIdx.x == 0 && threadIdx.x == 0) *status = 0;
 
