@@ -170,6 +170,8 @@ struct QuantCtl {
     int* sticky;            // device-wide sticky status word, or nullptr
     uint64_t wait_limit_ns;
     int starve;             // test hook: the producer of every CTA withholds its first row group
+    int feed_lanes;         // > 0: a barrier pair per row slot, fed by this many lanes of the producer warp (slot r by
+                            // lane r % feed_lanes); 0: a barrier pair per stage, fed by lane 0
 };
 
 __device__ __forceinline__ void bulk_load_row(uint32_t smem_dst, const void* gsrc, uint32_t bytes, uint32_t bar) {
@@ -196,22 +198,31 @@ quant_rows_staged_kernel(const __nv_bfloat16* __restrict__ x, int64_t ld, int ro
     uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t row_bytes = static_cast<uint32_t>(K) * 2u;
     const uint32_t stage_bytes = RPS * row_bytes;
-    // after the ring: full[num_stages], empty[num_stages], partial maxima, abort flag
+    // after the ring: full[num_stages][BPS], empty[num_stages][BPS], partial maxima, abort flag. With ROW_BARS
+    // every row slot of a stage has its own pair of barriers: a row is worked on as soon as it has landed and handed
+    // back as soon as its warps are done with it, so neither the first row of a launch nor the last one waits for the
+    // others of its stage. The launcher keeps one pair per stage where that measured faster (long rows in short rings).
+    const bool ROW_BARS = qc.feed_lanes > 0;
+    const int BPS = ROW_BARS ? RPS : 1;
     const uint32_t bars = base + num_stages * stage_bytes;
-    auto full_bar = [&](int s) { return bars + 8u * s; };
-    auto empty_bar = [&](int s) { return bars + 8u * (num_stages + s); };
-    float* s_red = reinterpret_cast<float*>(base_ptr + num_stages * stage_bytes + 16 * num_stages);
+    const int num_slots = num_stages * BPS;
+    auto full_bar = [&](int s, int slot) { return bars + 8u * (s * BPS + (ROW_BARS ? slot : 0)); };
+    auto empty_bar = [&](int s, int slot) { return bars + 8u * (num_slots + s * BPS + (ROW_BARS ? slot : 0)); };
+    float* s_red = reinterpret_cast<float*>(base_ptr + num_stages * stage_bytes + 16 * num_stages * RPS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(s_red + SG_WARPS);
     __shared__ int dummy_status;
     const WaitCtl ctl{abort_flag, status != nullptr ? status : &dummy_status, qc.sticky, qc.wait_limit_ns};
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int i = threadIdx.x; i < num_slots; i += SG_THREADS) {
+        mbar_init(bars + 8u * i, 1);                          // full: the producer's arrival with the row's byte count
+        mbar_init(bars + 8u * (num_slots + i), ROW_BARS ? WPR : SG_WARPS);    // empty: the warps of the row / stage
+    }
     if (threadIdx.x == 0) {
-        for (int s = 0; s < num_stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), SG_WARPS); }
         *abort_flag = 0;
         dummy_status = 0;
-        fence_mbar_init();
     }
+    fence_mbar_init();
     __syncthreads();
     // This kernel may itself have been launched early, behind a kernel that allowed it (programmatic dependent
     // launch): everything above touched shared memory only; global memory is touched after that kernel is complete.
@@ -222,24 +233,39 @@ quant_rows_staged_kernel(const __nv_bfloat16* __restrict__ x, int64_t ld, int ro
 
     if (warp == SG_WARPS) {
         // ---------------------------------------------------------------- producer
-        if (lane == 0) {
+        // ROW_BARS: the row slots of every stage are dealt to feed_lanes lanes (short rows: one lane per slot, so
+        // that the waits for the slots overlap instead of queueing behind one thread; longer rows: one lane, whose
+        // copies leave one after another and keep the rows of a stage staggered); otherwise lane 0 feeds whole stages.
+        const int feed_lanes = ROW_BARS ? qc.feed_lanes : 1;
+        if (lane < feed_lanes) {
             int stage = 0;
             uint32_t phase = 0;
             bool withhold = qc.starve != 0;
             for (int g = blockIdx.x; g < total_groups; g += gridDim.x) {
-                if (!mbar_wait(empty_bar(stage), phase ^ 1u, ctl, 1, kStatusTimeout)) break;
-                if (withhold) {
-                    // test hook: nothing is posted for this stage, so the consumers' bounded wait on it runs out
-                    withhold = false;
-                    if (++stage == num_stages) { stage = 0; phase ^= 1u; }
-                    continue;
-                }
                 const int r0 = g * RPS;
                 const int nr = min(RPS, rows - r0);
-                mbar_arrive_expect_tx(full_bar(stage), nr * row_bytes);
-                for (int r = 0; r < nr; ++r)
-                    bulk_load_row(base + stage * stage_bytes + r * row_bytes, x + static_cast<int64_t>(r0 + r) * ld,
-                                  row_bytes, full_bar(stage));
+                if (ROW_BARS) {
+                    bool go = true;
+                    for (int r = lane; r < nr; r += feed_lanes) {
+                        if (!mbar_wait(empty_bar(stage, r), phase ^ 1u, ctl, 1, kStatusTimeout)) { go = false; break; }
+                        if (!withhold) {
+                            mbar_arrive_expect_tx(full_bar(stage, r), row_bytes);
+                            bulk_load_row(base + stage * stage_bytes + r * row_bytes,
+                                          x + static_cast<int64_t>(r0 + r) * ld, row_bytes, full_bar(stage, r));
+                        }
+                    }
+                    if (!go) break;
+                } else {
+                    if (!mbar_wait(empty_bar(stage, 0), phase ^ 1u, ctl, 1, kStatusTimeout)) break;
+                    if (!withhold) {
+                        mbar_arrive_expect_tx(full_bar(stage, 0), nr * row_bytes);
+                        for (int r = 0; r < nr; ++r)
+                            bulk_load_row(base + stage * stage_bytes + r * row_bytes,
+                                          x + static_cast<int64_t>(r0 + r) * ld, row_bytes, full_bar(stage, 0));
+                    }
+                }
+                // test hook (withhold): nothing is posted for the first group, so the consumers' bounded wait runs out
+                withhold = false;
                 if (++stage == num_stages) { stage = 0; phase ^= 1u; }
             }
         }
@@ -256,7 +282,7 @@ quant_rows_staged_kernel(const __nv_bfloat16* __restrict__ x, int64_t ld, int ro
             // load: the value may have been written by the kernel ahead while this one was already resident)
             float amax_given = 0.f;
             if (GIVEN && row < rows) amax_given = __ldcg(amax_in + row);
-            if (ok && !mbar_wait(full_bar(stage), phase, ctl, 2, kStatusTimeout)) ok = false;
+            if (ok && (row < rows || !ROW_BARS) && !mbar_wait(full_bar(stage, slot), phase, ctl, 2, kStatusTimeout)) ok = false;
             ok = __all_sync(0xffffffffu, ok) != 0;
             const bool live = ok && row < rows;
             const uint4* srow = reinterpret_cast<const uint4*>(base_ptr + stage * stage_bytes + slot * row_bytes);
@@ -310,7 +336,7 @@ quant_rows_staged_kernel(const __nv_bfloat16* __restrict__ x, int64_t ld, int ro
                 }
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(empty_bar(stage));    // this warp is done with the stage
+            if (lane == 0 && (row < rows || !ROW_BARS)) mbar_arrive(empty_bar(stage, slot));    // done with its row / the stage
             if (++stage == num_stages) { stage = 0; phase ^= 1u; }
         }
     }
@@ -525,7 +551,7 @@ cudaError_t launch_staged(const __nv_bfloat16* x, int64_t ld, int rows, int K, i
     if (num_stages < 2 && 2 * stage_bytes + 1024 <= SG_SMEM_MAX) num_stages = 2;
     // the ring indices of the kernel wrap at num_stages: a ring of fewer than two stages must never be launched
     if (num_stages < 2) return cudaErrorInvalidConfiguration;
-    const int smem = num_stages * stage_bytes + 16 * num_stages + SG_WARPS * 4 + 16 + 128;
+    const int smem = num_stages * stage_bytes + 16 * num_stages * RPS + SG_WARPS * 4 + 16 + 128;
     static PerDeviceOnce smem_opt_in;
     const cudaError_t attr_err = smem_opt_in.run([] {
         cudaError_t e = cudaFuncSetAttribute(quant_rows_staged_kernel<WPR, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -542,7 +568,18 @@ cudaError_t launch_staged(const __nv_bfloat16* x, int64_t ld, int rows, int K, i
     const int cap = ctas_per_sm * sm_count();
     const int grid = groups < cap ? groups : cap;
     const float* none = nullptr;
-    const QuantCtl qc{status, sticky_status_word(), wait_limit_ns(), starve_mode() == kStarveQuant ? 1 : 0};
+    // Barrier granularity and the lanes that feed the ring, from timings of back-to-back launches on B200: a pair of
+    // barriers per row wherever the ring is long (one CTA per SM) or the rows are short; per stage for rows above
+    // 4 KB in the half-size rings of two CTAs per SM. Short rows want a feeding lane per row slot (one thread's
+    // wait-and-issue per row is what limits them), rows of 6 KB and more one or two.
+    const int row_bytes = K * 2;
+    int feed_lanes;
+    if (row_bytes <= 2048)      feed_lanes = RPS;
+    else if (row_bytes <= 4096) feed_lanes = 4;
+    else if (ctas_per_sm == 2)  feed_lanes = 0;
+    else                        feed_lanes = WPR <= 4 ? 2 : 1;
+    if (feed_lanes > RPS) feed_lanes = RPS;
+    const QuantCtl qc{status, sticky_status_word(), wait_limit_ns(), starve_mode() == kStarveQuant ? 1 : 0, feed_lanes};
     if (amax != nullptr)
         return launch_pdl(quant_rows_staged_kernel<WPR, false, true>, grid, SG_THREADS, smem, st, x, ld, rows, K, q, s, qc, num_stages, none, amax);
     if (mult != nullptr)
