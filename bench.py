@@ -30,8 +30,8 @@ INT8_PEAK_TOPS = 4500.0            # B200 datasheet, dense INT8
 # program on that workload, averaged over the workload's GEMM launches), with the summary it is taken from. Workloads
 # that were not captured have no entry: the bench line then says null and why.
 NCU_GEMM_DRAM_TRAFFIC = {
-    "c4": {"bytes_per_launch": 126.65e6, "profile": "profiles/gemm_tc_kernel_c4_mlp.md",
-           "note": "mean of the up (124.8 MB) and down (128.5 MB) launches; algorithmic bytes 165.2 / 122.7 MB"},
+    "c4": {"bytes_per_launch": 126.3e6, "profile": "profiles/gemm_tc_kernel_c4_mlp.md",
+           "note": "mean of the up (124.8 MB) and down (127.7 MB) launches; algorithmic bytes 165.2 / 122.7 MB"},
     "paper": {"bytes_per_launch": None, "profile": "profiles/gemm_tc_kernel_paper_llm_proj_ksplit.md",
               "note": "only the llm-proj launch was captured (1.42 GB against 502 MB algorithmic); no per-workload mean"},
 }
