@@ -583,22 +583,32 @@ def main():
 
         if not args.no_extras:
             # ---- end to end through the host-buffer entry point: pinned host activations in, host result out
+            # Two copies of every linear's buffers (host and device) where the run has two input sets: consecutive
+            # steps then share nothing, and a step's uploads need not wait for the previous step's downloads.
+            copies = min(2, len(sets))
             e2e_sets = []
-            for L in sets[0]:
-                spec = L["spec"]
-                e2e_sets.append({"L": L, "A_host": L["A"].cpu().pin_memory(),
-                                 "out_host": torch.empty((spec.M, spec.N), dtype=torch.bfloat16).pin_memory(),
-                                 "d_A": torch.empty_like(L["A"])})
+            for c in range(copies):
+                row = []
+                for L in sets[c]:
+                    spec = L["spec"]
+                    row.append({"L": L, "A_host": L["A"].cpu().pin_memory(),
+                                "out_host": torch.empty((spec.M, spec.N), dtype=torch.bfloat16).pin_memory(),
+                                "d_A": torch.empty_like(L["A"])})
+                e2e_sets.append(row)
 
-            # the linears of a step go to two streams in turn, so that one linear's download overlaps the next one's
-            # upload (PCIe is full duplex); each linear has its own workspace, device and host buffers
+            # the linears of a step go to two streams in turn (and the next step to two others), so that one linear's
+            # download overlaps another one's upload (PCIe is full duplex); every call in flight has its own
+            # workspace, device and host buffers
             main_stream = torch.cuda.current_stream(dev)
-            side = [torch.cuda.Stream(dev), torch.cuda.Stream(dev)]
+            side = [torch.cuda.Stream(dev) for _ in range(2 * copies)]
+            e2e_calls = [0]
 
             def e2e_step():
-                for i, e in enumerate(e2e_sets):
+                c = e2e_calls[0] % copies
+                e2e_calls[0] += 1
+                for i, e in enumerate(e2e_sets[c]):
                     L = e["L"]
-                    with torch.cuda.stream(side[i % 2]):
+                    with torch.cuda.stream(side[2 * c + i % 2]):
                         w8.int8_linear_fused_host(e["A_host"], e["d_A"], L["qw"], L["s_ch"], L["bias"], L["out"], e["out_host"], L["ws"])
 
             def fork():
@@ -633,7 +643,8 @@ def main():
             line["e2e"] = {"value": ops_per_step / e2e_sec / 1e12, "unit": "TOPS",
                            "h2d_bytes_per_step": sum(2 * s.M * s.K for s in specs),
                            "d2h_bytes_per_step": sum(2 * s.M * s.N for s in specs), "ms_per_step": e2e_sec * 1e3,
-                           "entry": "int8_linear_fused_host (pinned host bf16 in, pinned host bf16 out), linears alternating over two streams"}
+                           "entry": "int8_linear_fused_host (pinned host bf16 in, pinned host bf16 out), linears alternating over "
+                                    f"{len(side)} streams, {copies} sets of buffers"}
 
             # ---- context on the same box: library bf16 matmul and library int8 matmul on the same shapes
             ctx = []
