@@ -483,6 +483,28 @@ def test_k_split_from_bf16_automatic_choice():
 
 # ------------------------------------------------------------------------------- quantizer fused into its producer
 
+# Shapes that between them reach every way the staged quantizer runs its ring: a barrier pair per row slot fed by
+# 16 / 4 / 2 / 1 producer lanes or a pair per stage, one or two CTAs per SM (two from 8 row groups per SM on), a last
+# group with fewer rows than a stage has slots.
+@pytest.mark.parametrize("M,K", [(19003, 1024), (37889, 512), (10007, 2048), (9497, 1536), (9481, 3072), (4737, 4096),
+                                 (4740, 6144), (2369, 12288), (1185, 16384), (9473, 16)])
+def test_act_quantizer_every_ring_variant_against_oracle(M, K):
+    rng = np.random.default_rng(M + K)
+    scale = rng.choice(np.array([0.01, 1.0, 50.0], dtype=np.float32), size=(M, 1))
+    A = torch.from_numpy(rng.standard_normal((M, K), dtype=np.float32) * scale).to(torch.bfloat16)
+    A[int(rng.integers(0, M))] = 0
+    bits = synth.bf16_bits(A)
+    qa_ref, s_ref = oracle.quantize_act_per_token(bits)
+    dA = A.to(DEV)
+    qa, s = w8.int8_quantize_act_per_token(dA)
+    assert np.array_equal(s.cpu().numpy().view(np.uint32), s_ref.view(np.uint32))
+    assert np.array_equal(qa.cpu().numpy(), qa_ref)
+    qa1, s1 = w8.int8_quantize_act_per_token_given_absmax(dA, torch.from_numpy(oracle.row_absmax_bf16(bits)).to(DEV))
+    assert np.array_equal(s1.cpu().numpy().view(np.uint32), s_ref.view(np.uint32))
+    assert np.array_equal(qa1.cpu().numpy(), qa_ref)
+    assert w8.int8_sticky_status(clear=True) == 0
+
+
 @pytest.mark.parametrize("M,K", [(1, 16), (33, 2048), (300, 3072), (40, 12288), (3, 40000), (6, 53248), (2, 66000)])
 def test_one_pass_quantizer_with_the_absmax_handed_in(M, K):
     spec = synth.LinearSpec(f"q1p{M}x{K}", M, K, 8, outlier_frac=0.01 if K >= 256 else 0.0)
@@ -861,7 +883,8 @@ def test_gemm_wait_runs_out_and_the_kernel_returns(short_waits, M, K, N, cfg):
     assert w8.int8_sticky_status(clear=True) == 0
 
 
-@pytest.mark.parametrize("M,K", [(300, 1024), (40, 12288), (6, 53248)])
+# row-slot barriers fed by 16 lanes / by one lane, one-row stages, and stage barriers (two CTAs per SM, rows above 4 KB)
+@pytest.mark.parametrize("M,K", [(300, 1024), (40, 12288), (6, 53248), (9481, 3072)])
 def test_quantizer_wait_runs_out_and_the_kernel_returns(short_waits, M, K):
     spec = synth.LinearSpec(f"toq{M}x{K}", M, K, 8)
     A = synth.make_activations(spec)
