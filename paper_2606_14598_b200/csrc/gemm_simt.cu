@@ -57,7 +57,13 @@ gemm_simt_kernel(const int8_t* qa, int64_t lda_q, const float* s_tok,
 #pragma unroll
         for (int j = 0; j < NPW; ++j) w[j] = __ldg(reinterpret_cast<const uint4*>(wrow[j] + k));
 #pragma unroll
-        for (int i = 0; i < MB; ++i) a[i] = __ldcg(reinterpret_cast<const uint4*>(arow[i] + k));
+        // Coherent loads (the quantizer ahead may have written these rows while this kernel was already resident).
+        // One or two rows: plain, L1-cached ones, since every warp of the CTA re-reads them and nothing of them was
+        // touched before the wait above, so no line in this SM's L1 can predate the quantizer's writes (12.1 against
+        // 14.3-18.7 us at M = 1-2 with L2-only loads); more rows: L2-only loads, which leave L1 to the weight
+        // stream (15.5 against 17.2 us at M = 4).
+        for (int i = 0; i < MB; ++i)
+            a[i] = MB <= 2 ? *reinterpret_cast<const uint4*>(arow[i] + k) : __ldcg(reinterpret_cast<const uint4*>(arow[i] + k));
 #pragma unroll
         for (int i = 0; i < MB; ++i)
 #pragma unroll
