@@ -294,6 +294,21 @@ uint64_t int8_debug_set_wait_limit_ns(uint64_t limit_ns);
 int int8_debug_set_starve(int mode);
 
 /*
+ * Test-only choice of the one-kernel path (Method, "The fused kernel": the paper's kernel leaves the per-token
+ * quantizer to a launch of its own; for bf16 problems of at most 128 tokens and K <= 1024 this library can run
+ * quantizer, GEMM and epilogue in one launch, the CTAs of a cluster sharing the quantizer's work; results, workspace contents
+ * and status behaviour are those of the two-kernel path, bit for bit).
+ *   -1  chosen from the shape (default: more than 8 and at most 128 tokens, K <= 1024, N <= 1024, at most 16 Ki
+ *       elements of A per CTA of a cluster of up to four; never while a configuration is forced or with SmoothQuant
+ *       factors)
+ *    0  never
+ *    1  wherever the kernel can run (1 <= M <= 128, K <= 1024), forced configurations notwithstanding
+ * Returns the previous mode, -2 for an unknown one. With mode 1 and int8_debug_set_starve(1) the kernel's only wait
+ * (for its MMAs) runs out. Process-wide, like the other test controls.
+ */
+int int8_debug_set_small_path(int mode);
+
+/*
  * Force a kernel configuration for sweeps and tests. -1 = choose from the shape; -2 = choose from the shape
  * but never cut tiles along K; id = that configuration; id + 0x100 = that configuration, never cut along K.
  * For the configuration whose tiles are two sub-tiles side by side, bits 12-19, if not zero, are 1 + the number of
@@ -314,7 +329,9 @@ int int8_linear_force_config(int config_id);
 int int8_linear_plan(int64_t M, int64_t N, int64_t K, int a_dtype, size_t workspace_bytes,
                      int* config_id, int* cta_groups, int* split_tiles, int* split_parts);
 
-/* Number of kernel configurations, and a short description of one (NULL if out of range). */
+/* Number of kernel configurations that can be forced, and a short description of one (NULL if out of range). The id
+ * int8_linear_num_configs() itself names the one-kernel path for small problems, which int8_linear_plan reports where
+ * the shape selects it and which cannot be forced through int8_linear_force_config. */
 int int8_linear_num_configs(void);
 const char* int8_linear_config_name(int config_id);
 

@@ -19,7 +19,7 @@ _BINDING_NAMES = (
     "int8_quantize_act_per_token", "int8_quantize_weight_per_channel", "num_configs",
     "int8_quantize_act_per_token_smooth", "int8_quantize_weight_per_channel_smooth", "int8_linear_fused_smooth",
     "status_string", "int8_linear_workspace_min_bytes", "int8_linear_plan", "int8_sticky_status",
-    "debug_set_wait_limit_ns", "debug_set_starve", "gemm_clock_stamps", "int8_linear_fused_rowmax",
+    "debug_set_wait_limit_ns", "debug_set_starve", "debug_set_small_path", "gemm_clock_stamps", "int8_linear_fused_rowmax",
     "int8_quantize_act_per_token_given_absmax",
 )
 

@@ -27,7 +27,7 @@ EXPORTS = (
     "int8_check_status", "int8_linear_force_config", "int8_linear_num_configs", "int8_linear_config_name",
     "int8_status_string", "int8_linear_fused_static", "int8_quantize_weight_per_channel_smooth",
     "int8_quantize_act_per_token_smooth", "int8_linear_fused_smooth", "int8_linear_workspace_min_bytes", "int8_linear_plan",
-    "int8_sticky_status", "int8_debug_set_wait_limit_ns", "int8_debug_set_starve",
+    "int8_sticky_status", "int8_debug_set_wait_limit_ns", "int8_debug_set_starve", "int8_debug_set_small_path",
     "int8_linear_fused_rowmax", "int8_quantize_act_per_token_given_absmax", "int8_linear_fused_given_absmax",
 )
 
@@ -79,6 +79,8 @@ _lib.int8_debug_set_wait_limit_ns.argtypes = [ctypes.c_uint64]
 _lib.int8_debug_set_wait_limit_ns.restype = ctypes.c_uint64
 _lib.int8_debug_set_starve.argtypes = [_int]
 _lib.int8_debug_set_starve.restype = _int
+_lib.int8_debug_set_small_path.argtypes = [_int]
+_lib.int8_debug_set_small_path.restype = _int
 _lib.int8_linear_force_config.argtypes = [_int]
 _lib.int8_linear_force_config.restype = _int
 _lib.int8_linear_num_configs.argtypes = []
@@ -396,6 +398,11 @@ def debug_set_wait_limit_ns(limit_ns: int) -> int:
 def debug_set_starve(mode: int) -> int:
     """Test-only: 1 = the GEMM's producer withholds a stage, 2 = the quantizer's producer does; 0 = off."""
     return int(_lib.int8_debug_set_starve(int(mode)))
+
+
+def debug_set_small_path(mode: int) -> int:
+    """Test-only: -1 = the one-kernel path where the shape calls for it (default), 0 = never, 1 = wherever it can run."""
+    return int(_lib.int8_debug_set_small_path(int(mode)))
 
 
 def gemm_clock_stamps(workspace: torch.Tensor):

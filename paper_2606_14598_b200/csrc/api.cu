@@ -14,12 +14,22 @@ namespace {
 using namespace w8a8;
 
 constexpr size_t kStatusBlock = 256;
-constexpr int kSkinnyM = 8;           // at or below this many tokens the weight-streaming path runs (measured: it wins
-                                      // up to 4-8 tokens, the tensor-core path from 16 on)
+// kSkinnyM (internal.h): at or below this many tokens the weight-streaming path runs (measured: it wins up to 4-8
+// tokens, the tensor-core path from 16 on)
 
 std::atomic<int> g_forced_config{-1};
 std::atomic<uint64_t> g_wait_limit_ns{2000000000ull};     // 2 s
 std::atomic<int> g_starve{0};
+std::atomic<int> g_small_mode{-1};
+
+// The one-kernel path takes bf16 activations without SmoothQuant factors; chosen by shape unless a test says otherwise.
+bool use_small_path(int a_dtype, const float* a_mult, int forced, int64_t M, int64_t N, int64_t K) {
+    if (a_dtype != W8A8_ACT_BF16 || a_mult != nullptr) return false;
+    const int mode = g_small_mode.load();
+    if (mode == 0) return false;
+    if (mode == 1) return small_fused_eligible(M, N, K);
+    return forced < 0 && small_fused_preferred(M, N, K);
+}
 
 // First time-out recorded by any kernel of this library on the device, kept until the host clears it. (The status
 // word of a workspace is reset by every call on that workspace; this one is not.) Zero when the module is loaded.
@@ -75,6 +85,7 @@ namespace w8a8 {
 
 uint64_t wait_limit_ns() { return g_wait_limit_ns.load(); }
 int starve_mode() { return g_starve.load(); }
+int small_path_mode() { return g_small_mode.load(); }
 
 int* sticky_status_word() {
     int dev = -1;
@@ -95,6 +106,11 @@ extern "C" {
 uint64_t int8_debug_set_wait_limit_ns(uint64_t limit_ns) {
     if (limit_ns == 0) limit_ns = 2000000000ull;
     return g_wait_limit_ns.exchange(limit_ns);
+}
+
+int int8_debug_set_small_path(int mode) {
+    if (mode < -1 || mode > 1) return -2;
+    return g_small_mode.exchange(mode);
 }
 
 int int8_debug_set_starve(int mode) {
@@ -132,6 +148,7 @@ int int8_linear_force_config(int config_id) { return g_forced_config.exchange(co
 int int8_linear_num_configs(void) { return tc_num_configs() + 1; }
 const char* int8_linear_config_name(int config_id) {
     if (config_id == tc_num_configs()) return "simt dp4a (skinny M / cross-check)";
+    if (config_id == tc_num_configs() + 1) return "one kernel: quantizer + tc 128x32 per CTA (small problems)";
     return tc_config_name(config_id);
 }
 
@@ -212,7 +229,10 @@ int int8_linear_plan(int64_t M, int64_t N, int64_t K, int a_dtype, size_t worksp
     // no device needed: the plan depends on the SM count only (148 is assumed when no device can be queried)
     const int forced = g_forced_config.load();
     TcPlan plan{};
-    if ((forced < 0 && M <= kSkinnyM) || (forced >= 0 && (forced & 0xff) == tc_num_configs())) {
+    if (use_small_path(a_dtype, nullptr, forced, M, N, K)) {
+        plan.config = tc_num_configs() + 1;
+        plan.groups = static_cast<int>((N + 31) / 32);
+    } else if ((forced < 0 && M <= kSkinnyM) || (forced >= 0 && (forced & 0xff) == tc_num_configs())) {
         plan.config = tc_num_configs();
     } else {
         plan = tc_plan(static_cast<int>(M), static_cast<int>(N), static_cast<int>(K), forced, workspace_bytes - base);
@@ -257,6 +277,19 @@ static int fused_impl(const void* A, int a_dtype, int64_t lda, const float* s_to
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     int* status = reinterpret_cast<int*>(ws);
     const int forced = g_forced_config.load();
+    if (use_small_path(a_dtype, a_mult, forced, M, N, K)) {
+        if (rowmax_out != nullptr && cudaMemsetAsync(rowmax_out, 0, static_cast<size_t>(M) * sizeof(float), st) != cudaSuccess)
+            return W8A8_ERR_CUDA;
+        GemmArgs g{};
+        g.rowmax = rowmax_out;
+        g.qw = qw; g.s_ch = s_ch; g.bias = bias; g.out = out_bf16; g.ldo = ldo;
+        g.M = static_cast<int>(M); g.N = static_cast<int>(N); g.K = static_cast<int>(K);
+        g.status = status;
+        size_t s_off, q_off;
+        offsets(M, &s_off, &q_off);
+        return launch_small_fused(A, lda, amax_in, g, reinterpret_cast<int8_t*>(ws + q_off),
+                                  reinterpret_cast<float*>(ws + s_off), st) == cudaSuccess ? W8A8_OK : W8A8_ERR_CUDA;
+    }
     const bool simt = (forced < 0 && M <= kSkinnyM) || (forced >= 0 && (forced & 0xff) == tc_num_configs());
     // whatever the workspace holds beyond the required part is scratch for the K-split of the partial wave
     const size_t scratch_off = int8_linear_workspace_min_bytes(M, N, K, a_dtype);

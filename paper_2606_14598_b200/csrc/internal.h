@@ -91,6 +91,18 @@ struct GemmArgs {
 };
 cudaError_t launch_gemm_simt(const GemmArgs& a, cudaStream_t st);
 
+// ---- small_fused.cu : quantizer, GEMM and epilogue in one kernel, for problems of at most 128 tokens and K <= 1024
+constexpr int kSkinnyM = 8;           // at or below this many tokens the weight-streaming path runs
+constexpr int64_t kSmallFusedMaxCtas = 32;                 // 32-channel CTAs the one-kernel path is chosen for (N <= 1024)
+constexpr int64_t kSmallFusedMaxElemsPerCta = 16 << 10;    // elements of A one of its CTAs may have to quantize
+bool small_fused_eligible(int64_t M, int64_t N, int64_t K);     // what the kernel can run
+bool small_fused_preferred(int64_t M, int64_t N, int64_t K);    // where it is chosen when nothing is forced
+// Writes the codes and scales to qa_out / s_tok_out as the two-kernel path does, the output to g.out.
+cudaError_t launch_small_fused(const void* A_bf16, int64_t lda, const float* amax_in, const GemmArgs& g, int8_t* qa_out,
+                               float* s_tok_out, cudaStream_t st);
+// Test-only: -1 = chosen by small_fused_preferred (default), 0 = never, 1 = wherever small_fused_eligible.
+int small_path_mode();
+
 // ---- gemm_tc.cu : tcgen05 path
 int tc_num_configs();
 const char* tc_config_name(int id);

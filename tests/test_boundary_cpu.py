@@ -75,8 +75,8 @@ def test_plan_of_the_benchmark_shapes():
     assert p["split_parts"] == 2 and p["groups"] == p["split_tiles"] * 2 <= 74, p
     assert w8.int8_linear_plan(4110, 4608, 4608, w8.ACT_BF16)["split_parts"] == 0       # shallow K: a cut would not pay
     assert w8.int8_linear_plan(2, 18432, 3072, w8.ACT_BF16)["config"] == w8.num_configs() - 1   # CUDA-core path
-    assert "128x128" in w8.int8_linear_plan(128, 256, 256, w8.ACT_BF16)["name"] or \
-           "256x128" in w8.int8_linear_plan(128, 256, 256, w8.ACT_BF16)["name"]
+    assert "128x128" in w8.int8_linear_plan(128, 256, 256, w8.ACT_INT8)["name"] or \
+           "256x128" in w8.int8_linear_plan(128, 256, 256, w8.ACT_INT8)["name"]
     # forcing a configuration cuts whenever it can; + 0x100 never cuts; -2 chooses freely but never cuts
     w8.force_config(pair)
     assert w8.int8_linear_plan(256, 512, 2048, w8.ACT_INT8, 64 << 20)["split_parts"] == 2
@@ -89,9 +89,31 @@ def test_plan_of_the_benchmark_shapes():
         w8.int8_linear_plan(4110, 4608, 53248, w8.ACT_BF16, 1024)                       # below the minimum
 
 
+def test_one_kernel_path_is_chosen_for_one_tile_problems_only():
+    """Host logic of the default mode: c1 and its like take the one-kernel path; larger or skinnier problems, forced
+    configurations and pre-quantized activations do not."""
+    ws_big = 1 << 30
+    name = lambda M, N, K, a=w8.ACT_BF16: w8.int8_linear_plan(M, N, K, a, ws_big)["name"]
+    assert "one kernel" in name(128, 256, 256)          # c1
+    assert "one kernel" in name(16, 1024, 512)
+    assert "one kernel" not in name(128, 256, 256, w8.ACT_INT8)
+    assert "one kernel" not in name(128, 1024, 1024)    # 32 Ki elements per CTA of a cluster of four
+    assert "one kernel" not in name(129, 256, 256)
+    assert "one kernel" not in name(64, 2048, 256)      # N > 1024
+    assert "one kernel" not in name(8, 256, 256)        # skinny: the weight-streaming kernel
+    assert "one kernel" not in name(2816, 3072, 3072)
+    w8.force_config(0)
+    try:
+        assert "one kernel" not in name(128, 256, 256)
+    finally:
+        w8.force_config(-1)
+
+
 def test_configs_are_listed():
     n = w8.num_configs()
-    assert n >= 2 and all(w8.config_name(i) for i in range(n)) and w8.config_name(n) is None
+    # ids below n can be forced; id n only appears in plans (the one-kernel path for small problems is chosen by shape)
+    assert n >= 2 and all(w8.config_name(i) for i in range(n)) and "one kernel" in w8.config_name(n)
+    assert w8.config_name(n + 1) is None
     assert w8.force_config(-1) == -1
 
 

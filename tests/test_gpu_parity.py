@@ -914,3 +914,86 @@ def test_quantizer_wait_runs_out_and_the_kernel_returns(short_waits, M, K):
     ref = oracle.linear_fused_bf16(synth.bf16_bits(A), qw_ref, s_ch_ref, None)
     assert_bf16_close(synth.bf16_bits(out.cpu()), ref["out"])
     assert w8.int8_sticky_status(clear=True) == 7
+
+
+# ------------------------------------------------------------------------------- one-kernel path for small problems
+
+@pytest.fixture
+def small_path():
+    """Yields a setter of the one-kernel path's mode; the default (chosen from the shape) is restored afterwards."""
+    yield w8.debug_set_small_path
+    w8.debug_set_small_path(-1)
+
+
+# K <= 256 / 512 / 1024 (one, two, four 16-byte units per lane) x clusters of 1, 2 and 4 CTAs (N <= 32, <= 64, more),
+# ragged M, N and K, a grid padded to whole clusters (N = 264: 9 CTAs -> 12), a single token, the largest shape
+@pytest.mark.parametrize("M,K,N", [(128, 256, 256), (100, 272, 264), (9, 16, 8), (77, 1008, 40), (1, 512, 96),
+                                   (128, 1024, 1024), (33, 640, 2048), (128, 128, 32), (64, 768, 4736), (17, 48, 56)])
+def test_one_kernel_path_against_oracle(small_path, M, K, N):
+    rng = np.random.default_rng(M * 7 + K + N)
+    A = torch.from_numpy(rng.standard_normal((M, K), dtype=np.float32)).to(torch.bfloat16)
+    if M > 2:
+        A[1] = 0                                   # an all-zero token
+    W = rng.standard_normal((N, K), dtype=np.float32) * np.float32(0.02)
+    bias = rng.standard_normal(N, dtype=np.float32) * np.float32(0.01)
+    qw_ref, s_ch_ref = oracle.quantize_weight_per_channel(W)
+    bits = synth.bf16_bits(A)
+    ref = oracle.linear_fused_bf16(bits, qw_ref, s_ch_ref, bias)
+    ref_nb = oracle.linear_fused_bf16(bits, qw_ref, s_ch_ref, None)
+    # activations as a view with a row stride, output into a wider buffer
+    A_wide = torch.zeros((M, K + 32), dtype=torch.bfloat16, device=DEV)
+    A_wide[:, :K] = A.to(DEV)
+    dA = A_wide[:, :K]
+    out_wide = torch.full((M, N + 16), 7.0, dtype=torch.bfloat16, device=DEV)
+    qw, s_ch = w8.int8_quantize_weight_per_channel(torch.from_numpy(W).to(DEV))
+    db = torch.from_numpy(bias).to(DEV)
+    ws = w8.alloc_workspace(M, N, K, w8.ACT_BF16, DEV)
+    small_path(1)
+    assert "one kernel" in w8.int8_linear_plan(M, N, K, w8.ACT_BF16, ws.numel())["name"]
+    ws.zero_()
+    out, rowmax = w8.int8_linear_fused_rowmax(dA, qw, s_ch, db, out=out_wide[:, :N], workspace=ws)
+    check_status(ws)
+    assert np.array_equal(synth.bf16_bits(out.cpu()), ref["out"])
+    assert torch.all(out_wide[:, N:] == 7.0)       # nothing written beyond the N columns
+    assert np.array_equal(rowmax.cpu().numpy(), oracle.row_absmax_bf16(ref["out"]))
+    # the workspace holds codes and scales, as after the two-kernel path
+    s_off, q_off = w8.int8_linear_workspace_offsets(M, K)
+    assert np.array_equal(ws[q_off:q_off + M * K].view(torch.int8).view(M, K).cpu().numpy(), ref["qa"])
+    assert np.array_equal(ws[s_off:s_off + 4 * M].view(torch.float32).cpu().numpy().view(np.uint32), ref["s_tok"].view(np.uint32))
+    # without bias; with the absmax of every row handed in (one-pass quantizer inside the kernel)
+    out_nb = w8.int8_linear_fused(dA, qw, s_ch, None, workspace=ws)
+    check_status(ws)
+    assert np.array_equal(synth.bf16_bits(out_nb.cpu()), ref_nb["out"])
+    amax = torch.from_numpy(oracle.row_absmax_bf16(bits)).to(DEV)
+    out_g, _ = w8.int8_linear_fused_rowmax(dA, qw, s_ch, db, workspace=ws, rowmax_in=amax)
+    check_status(ws)
+    assert np.array_equal(synth.bf16_bits(out_g.cpu()), ref["out"])
+    # and the two-kernel path gives the same bits on the same call
+    small_path(0)
+    assert "one kernel" not in w8.int8_linear_plan(M, N, K, w8.ACT_BF16, ws.numel())["name"]
+    out2 = w8.int8_linear_fused(dA, qw, s_ch, db, workspace=ws)
+    check_status(ws)
+    assert np.array_equal(synth.bf16_bits(out2.cpu()), ref["out"])
+    assert w8.int8_sticky_status(clear=True) == 0
+
+
+def test_one_kernel_path_wait_runs_out_and_the_kernel_returns(short_waits, small_path):
+    """The MMA thread never commits (nothing invalid is touched): the epilogue warps' wait runs out after 3 ms, TMEM is
+    freed, the kernel returns and the status word says so; the next call on the same workspace is exact again."""
+    M, K, N = 128, 256, 256
+    spec, A, qw, s_ch, bias, ref = _timeout_case(M, K, N)
+    ws = w8.alloc_workspace(M, N, K, w8.ACT_BF16, DEV)
+    small_path(1)
+    w8.int8_sticky_status(clear=True)
+    w8.debug_set_starve(1)
+    w8.int8_linear_fused(A, qw, s_ch, bias, workspace=ws)
+    w8.debug_set_starve(0)
+    torch.cuda.synchronize()                          # returns: the kernel did not hang
+    raw_word = int(ws[:4].view(torch.int32).item())
+    assert raw_word & 0xff == 7 and (raw_word >> 8) == 4, hex(raw_word)
+    assert w8.int8_check_status(ws) == 7
+    out = w8.int8_linear_fused(A, qw, s_ch, bias, workspace=ws)
+    assert w8.int8_check_status(ws) == 0
+    assert np.array_equal(synth.bf16_bits(out.cpu()), ref["out"])
+    assert w8.int8_sticky_status(clear=True) == 7
+    assert w8.int8_sticky_status(clear=True) == 0
