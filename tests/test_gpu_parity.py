@@ -997,3 +997,28 @@ def test_one_kernel_path_wait_runs_out_and_the_kernel_returns(short_waits, small
     assert np.array_equal(synth.bf16_bits(out.cpu()), ref["out"])
     assert w8.int8_sticky_status(clear=True) == 7
     assert w8.int8_sticky_status(clear=True) == 0
+
+
+def test_one_kernel_path_random_small_shapes(small_path):
+    """200 seeded random shapes (M <= 128, K <= 1024, N <= 2400, with and without bias, an all-zero token) through the
+    one-kernel path: output, row maxima and the codes left in the workspace against the oracle, bit for bit."""
+    small_path(1)
+    for seed in range(200):
+        rng = np.random.default_rng(9000 + seed)
+        M, K, N = int(rng.integers(1, 129)), 16 * int(rng.integers(1, 65)), 8 * int(rng.integers(1, 300))
+        A = torch.from_numpy(rng.standard_normal((M, K), dtype=np.float32) * np.float32(rng.choice([0.05, 1.0, 30.0]))).to(torch.bfloat16)
+        if M > 3:
+            A[int(rng.integers(0, M))] = 0
+        W = rng.standard_normal((N, K), dtype=np.float32) * np.float32(0.02)
+        bias = rng.standard_normal(N, dtype=np.float32) * np.float32(0.01) if rng.integers(0, 2) else None
+        qw_ref, s_ch_ref = oracle.quantize_weight_per_channel(W)
+        ref = oracle.linear_fused_bf16(synth.bf16_bits(A), qw_ref, s_ch_ref, bias)
+        qw, s_ch = w8.int8_quantize_weight_per_channel(torch.from_numpy(W).to(DEV))
+        ws = w8.alloc_workspace(M, N, K, w8.ACT_BF16, DEV)
+        out, rowmax = w8.int8_linear_fused_rowmax(A.to(DEV), qw, s_ch, None if bias is None else torch.from_numpy(bias).to(DEV), workspace=ws)
+        check_status(ws)
+        assert np.array_equal(synth.bf16_bits(out.cpu()), ref["out"]), (M, K, N)
+        assert np.array_equal(rowmax.cpu().numpy(), oracle.row_absmax_bf16(ref["out"])), (M, K, N)
+        s_off, q_off = w8.int8_linear_workspace_offsets(M, K)
+        assert np.array_equal(ws[q_off:q_off + M * K].view(torch.int8).view(M, K).cpu().numpy(), ref["qa"]), (M, K, N)
+    assert w8.int8_sticky_status(clear=True) == 0
