@@ -128,9 +128,11 @@ void int8_linear_workspace_offsets(int64_t M, int64_t K, size_t* s_tok_offset, s
  *                  int8_linear_workspace_min_bytes(); two calls that may overlap on the device
  *                  need distinct workspaces
  * Requires K % 16 == 0, N % 8 == 0, K <= W8A8_K_MAX. The kernel configuration
- * (tile shape, pipeline depth, skinny-M path) is chosen from (M,N,K); the
+ * (tile shape, pipeline depth, skinny-M path, one kernel instead of two for
+ * bf16 problems of about one tile) is chosen from (M,N,K); the
  * paper's per-shape autotuning ("Why autotuning is load-bearing") is replaced
- * by a static per-shape table.
+ * by a static per-shape table. Whatever is chosen, outputs and the codes and
+ * scales left in the workspace are the same bit for bit.
  */
 int int8_linear_fused(const void* A, int a_dtype, int64_t lda, const float* s_tok_in,
                       const int8_t* qw, const float* s_ch, const float* bias,
