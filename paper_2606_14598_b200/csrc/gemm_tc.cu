@@ -837,11 +837,13 @@ TcPlan plan_config(int id, int M, int N, int K, bool allow_split, bool only_if_f
         const size_t need = kCounterBytes + static_cast<size_t>(rest) * c.cg * bn * BM * sizeof(int32_t);
         if (parts < 2 || need > scratch_bytes) parts = 1;
     }
-    // A partial wave that is left whole runs its tiles faster than the full-wave rate (measured ~0.72 of the tile
-    // time with few SMs active: the operand traffic of a full wave is what holds the rate down); a wave cut along K
+    // A partial wave that is left whole runs its tiles faster than the full-wave rate, since the operand traffic of a
+    // full wave is what holds the rate down: measured 0.68-0.78 of the tile time with a third of the SMs active for
+    // single CTAs, whose full-wave rate suffers most from that traffic, and 0.86-0.97 for CTA pairs. A wave cut along K
     // keeps every SM busy and pays ~10 us for zeroing the slabs, the reductions, the pipeline refill and the read-back.
     const double tile_us = 2.0 * BM * bn * static_cast<double>(K) / 20.3e6 / c.eff;
-    const double whole_rest_us = tile_us * (0.72 + 0.28 * rest / max_groups);
+    const double few = c.cg == 1 ? 0.66 : 0.85;
+    const double whole_rest_us = tile_us * (few + (1.0 - few) * rest / max_groups);
     const double split_rest_us = tile_us / parts + 10.0;
     if (parts > 1 && only_if_faster && split_rest_us >= whole_rest_us) parts = 1;
     double est = fixed_us + whole_waves * tile_us;
