@@ -56,6 +56,7 @@ def measured_peaks():
 SAMPLER_SRC = r"""
 import json, sys, time
 idx, period = sys.argv[1], float(sys.argv[2])
+sys.stdout = open(sys.argv[3], "a", buffering=1)
 import pynvml as nv
 nv.nvmlInit()
 h = nv.nvmlDeviceGetHandleByIndex(int(idx)) if idx.isdigit() else nv.nvmlDeviceGetHandleByUUID(idx)
@@ -89,17 +90,28 @@ class ClockSampler:
     def __init__(self, index: int, period_s: float = 0.002):
         import subprocess
         self.samples, self.power, self.reasons = [], [], set()
-        self.max_mhz, self.t0, self.t1, self.proc = None, None, None, None
+        self.max_mhz, self.t0, self.t1, self.proc, self.out = None, None, None, None, None
         visible = os.environ.get("CUDA_VISIBLE_DEVICES")
         tok = str(index)
         if visible:
             ids = [v for v in visible.split(",") if v.strip() != ""]
             tok = ids[index] if index < len(ids) else ids[0]
         try:
-            self.proc = subprocess.Popen([sys.executable, "-c", SAMPLER_SRC, tok, str(period_s)], stdout=subprocess.PIPE,
-                                         stderr=subprocess.DEVNULL, text=True)
-            first = self.proc.stdout.readline()            # the sampler is up once it has printed the maximum clock
-            self.max_mhz = json.loads(first)["max_mhz"] if first else None
+            # the samples go to a temporary file: a pipe would fill up (64 KB, a second or two of samples)
+            # while nobody reads it and block the sampler for the rest of the run
+            import tempfile
+            fd, self.out = tempfile.mkstemp(prefix="w8a8_clocks_", suffix=".jsonl")
+            os.close(fd)
+            self.proc = subprocess.Popen([sys.executable, "-c", SAMPLER_SRC, tok, str(period_s), self.out],
+                                         stdout=subprocess.DEVNULL, stderr=subprocess.DEVNULL)
+            first, deadline = "", time.time() + 20.0
+            while time.time() < deadline and self.proc.poll() is None:      # up once it has printed the maximum clock
+                with open(self.out) as f:
+                    first = f.readline()
+                if first.endswith("\n"):
+                    break
+                time.sleep(0.02)
+            self.max_mhz = json.loads(first)["max_mhz"] if first.endswith("\n") else None
             if self.max_mhz is None:
                 raise RuntimeError("no answer from the sampler")
         except Exception as e:          # NVML missing: report that no clocks were sampled
@@ -111,6 +123,12 @@ class ClockSampler:
             self.proc.kill()
             self.proc.wait()
             self.proc = None
+        if self.out is not None:
+            try:
+                os.unlink(self.out)
+            except OSError:
+                pass
+            self.out = None
 
     def __enter__(self):
         self.t0 = time.time()
@@ -122,9 +140,12 @@ class ClockSampler:
             return
         time.sleep(0.01)
         self.proc.kill()
-        out, _ = self.proc.communicate()
+        self.proc.wait()
         self.proc = None
-        for ln in out.splitlines():
+        with open(self.out) as f:
+            lines = f.read().splitlines()
+        self.close()
+        for ln in lines:
             try:
                 d = json.loads(ln)
             except Exception:
@@ -431,7 +452,9 @@ def main():
                   "note": "the step's int8_linear_fused calls issued one by one, timed right after the headline loop"}
     ops_all_ranks = wdist.sum_over_ranks(ops_per_step * args.steps, dev)
     tops = ops_all_ranks / sec / 1e12
-    launches = args.steps * sum(2 for _ in specs)      # quantizer + GEMM per linear
+    # quantizer + GEMM per linear; one launch where the shape takes the one-kernel path
+    launches = args.steps * sum(1 if "one kernel" in w8.int8_linear_plan(s_.M, s_.N, s_.K, w8.ACT_BF16)["name"] else 2
+                                for s_ in specs)
 
     line = {
         "metric": METRIC, "value": tops, "unit": "TOPS", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,

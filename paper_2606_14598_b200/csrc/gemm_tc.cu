@@ -797,7 +797,10 @@ TcPlan plan_config(int id, int M, int N, int K, bool allow_split, bool only_if_f
     }
     const int max_groups = sm_count() / c.cg;
     const int num_m = (M + BM * c.cg - 1) / (BM * c.cg);
-    const double fixed_us = 4.0;                       // launch, pipeline fill, last epilogue
+    // launch, pipeline fill, last epilogue; a pair pays for its cluster launch and for filling stages of twice the
+    // bytes (fitted on shapes of about one wave at K = 1536-3072: 3072 x 1536 x 1536 runs 8.9 us on single CTAs,
+    // 10.7 us on pairs with the same per-CTA tile)
+    const double fixed_us = c.cg == 1 ? 4.0 : 5.5;
     if (c.nsub == 2) {
         // ~20.3 int8 TOPS per SM for the 256 x 256 pair tile in whole waves; a unit = one column block of a row block
         const int num_nb = (N + c.bns - 1) / c.bns;
@@ -838,13 +841,15 @@ TcPlan plan_config(int id, int M, int N, int K, bool allow_split, bool only_if_f
         if (parts < 2 || need > scratch_bytes) parts = 1;
     }
     // A partial wave that is left whole runs its tiles faster than the full-wave rate, since the operand traffic of a
-    // full wave is what holds the rate down: measured 0.68-0.78 of the tile time with a third of the SMs active for
-    // single CTAs, whose full-wave rate suffers most from that traffic, and 0.86-0.97 for CTA pairs. A wave cut along K
-    // keeps every SM busy and pays ~10 us for zeroing the slabs, the reductions, the pipeline refill and the read-back.
+    // full wave is what holds the rate down: measured 0.68-0.80 of the tile time with a tenth to a third of the SMs
+    // active for single CTAs, whose full-wave rate suffers most from that traffic, and 0.86-0.97 for CTA pairs. A wave
+    // cut along K keeps every SM busy and pays for zeroing the slabs, the reductions, the pipeline refill and the
+    // read-back: 7-9 us measured on single CTAs with 128-column slabs, 11-12 us with 256-column ones and on pairs
+    // (M = 192-512, K = 8192, N = 264-2048).
     const double tile_us = 2.0 * BM * bn * static_cast<double>(K) / 20.3e6 / c.eff;
-    const double few = c.cg == 1 ? 0.66 : 0.85;
+    const double few = c.cg == 1 ? 0.72 : 0.85;
     const double whole_rest_us = tile_us * (few + (1.0 - few) * rest / max_groups);
-    const double split_rest_us = tile_us / parts + 10.0;
+    const double split_rest_us = tile_us / parts + (c.cg == 1 ? 5.5 + 6.0 * bn / 256 : 12.0);
     if (parts > 1 && only_if_faster && split_rest_us >= whole_rest_us) parts = 1;
     double est = fixed_us + whole_waves * tile_us;
     if (rest > 0) est += parts > 1 ? split_rest_us : whole_rest_us;
