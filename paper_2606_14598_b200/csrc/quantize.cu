@@ -132,7 +132,12 @@ quant_rows_staged_kernel(const __nv_bfloat16* __restrict__ x, int64_t ld, int ro
     grid_dep_wait();
     if (status != nullptr && blockIdx.x == 0 && threadIdx.x == 0) *status = 0;
 
-    const int total_groups = (rows + RPS - 1) / RPS;          // a group = the rows of one stage
+    // Every CTA takes a contiguous share of the rows, as even as the row count allows (not whole stages: with 2816 rows
+    // on 148 CTAs that is 20 rows each instead of 16 or 24), and walks it in groups of up to RPS rows (one stage each).
+    const int rows_per_cta = (rows + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
+    const int r_begin = min(rows, static_cast<int>(blockIdx.x) * rows_per_cta);
+    const int r_end = min(rows, r_begin + rows_per_cta);
+    const int my_groups = (r_end - r_begin + RPS - 1) / RPS;
 
     if (warp == SG_WARPS) {
         // ---------------------------------------------------------------- producer
@@ -144,9 +149,9 @@ quant_rows_staged_kernel(const __nv_bfloat16* __restrict__ x, int64_t ld, int ro
             int stage = 0;
             uint32_t phase = 0;
             bool withhold = qc.starve != 0;
-            for (int g = blockIdx.x; g < total_groups; g += gridDim.x) {
-                const int r0 = g * RPS;
-                const int nr = min(RPS, rows - r0);
+            for (int g = 0; g < my_groups; ++g) {
+                const int r0 = r_begin + g * RPS;
+                const int nr = min(RPS, r_end - r0);
                 if (ROW_BARS) {
                     bool go = true;
                     for (int r = lane; r < nr; r += feed_lanes) {
@@ -179,15 +184,15 @@ quant_rows_staged_kernel(const __nv_bfloat16* __restrict__ x, int64_t ld, int ro
         int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
-        for (int g = blockIdx.x; g < total_groups; g += gridDim.x) {
-            const int row = g * RPS + slot;
+        for (int g = 0; g < my_groups; ++g) {
+            const int row = r_begin + g * RPS + slot;
             // an absmax that is handed in is fetched while the row's bytes are still on their way (plain, coherent
             // load: the value may have been written by the kernel ahead while this one was already resident)
             float amax_given = 0.f;
-            if (GIVEN && row < rows) amax_given = __ldcg(amax_in + row);
-            if (ok && (row < rows || !ROW_BARS) && !mbar_wait(full_bar(stage, slot), phase, ctl, 2, kStatusTimeout)) ok = false;
+            if (GIVEN && row < r_end) amax_given = __ldcg(amax_in + row);
+            if (ok && (row < r_end || !ROW_BARS) && !mbar_wait(full_bar(stage, slot), phase, ctl, 2, kStatusTimeout)) ok = false;
             ok = __all_sync(0xffffffffu, ok) != 0;
-            const bool live = ok && row < rows;
+            const bool live = ok && row < r_end;
             const uint4* srow = reinterpret_cast<const uint4*>(base_ptr + stage * stage_bytes + slot * row_bytes);
             float amax = 0.f;
             if (GIVEN) {
@@ -239,7 +244,7 @@ quant_rows_staged_kernel(const __nv_bfloat16* __restrict__ x, int64_t ld, int ro
                 }
             }
             __syncwarp();
-            if (lane == 0 && (row < rows || !ROW_BARS)) mbar_arrive(empty_bar(stage, slot));    // done with its row / the stage
+            if (lane == 0 && (row < r_end || !ROW_BARS)) mbar_arrive(empty_bar(stage, slot));    // done with its row / the stage
             if (++stage == num_stages) { stage = 0; phase ^= 1u; }
         }
     }
@@ -469,7 +474,11 @@ cudaError_t launch_staged(const __nv_bfloat16* x, int64_t ld, int rows, int K, i
     });
     if (attr_err != cudaSuccess) return attr_err;
     const int cap = ctas_per_sm * sm_count();
-    const int grid = groups < cap ? groups : cap;
+    // few rows: CTAs of as little as a quarter of a stage's rows each, so that more SMs share the work (M = 512,
+    // K = 12288: 14.8 -> 5.5 us; M = 256, K = 3072: 6.8 -> 5.2 us, which is the host's launch rate)
+    const int rmin = RPS >= 4 ? RPS / 4 : 1;
+    const int want = (rows + rmin - 1) / rmin;
+    const int grid = want < cap ? want : cap;
     const float* none = nullptr;
     // Barrier granularity and the lanes that feed the ring, from timings of back-to-back launches on B200: a pair of
     // barriers per row wherever the ring is long (one CTA per SM) or the rows are short; per stage for rows above
