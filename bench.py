@@ -272,6 +272,8 @@ def main():
     ap.add_argument("--config", type=int, default=-1, help="force a kernel configuration (sweeps); -1 = from the shape")
     ap.add_argument("--repeats", type=int, default=0,
                     help="timed loops of --steps steps (0 = 7, enough for ten NVML samples over 20-step loops); the median is reported")
+    ap.add_argument("--small-path", default="auto", choices=["auto", "on", "off"],
+                    help="the one-kernel path for small problems: chosen from the shape / wherever it can run / never")
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         # no launcher: run one process per GPU ourselves (rank i on GPU i); the ranks meet through a rendezvous file
@@ -302,6 +304,7 @@ def main():
     specs = workload_specs(args)
     peaks = measured_peaks()
     w8.force_config(args.config)
+    w8.debug_set_small_path({"auto": -1, "on": 1, "off": 0}[args.small_path])
 
     # ---- set-up (untimed): seeded inputs, weights quantized on the device by the library
     sets = []

@@ -300,7 +300,7 @@ int int8_debug_set_starve(int mode);
  * quantizer to a launch of its own; for bf16 problems of at most 128 tokens and K <= 1024 this library can run
  * quantizer, GEMM and epilogue in one launch, the CTAs of a cluster sharing the quantizer's work; results, workspace contents
  * and status behaviour are those of the two-kernel path, bit for bit).
- *   -1  chosen from the shape (default: more than 8 and at most 128 tokens, K <= 1024, N <= 1024, at most 16 Ki
+ *   -1  chosen from the shape (default: more than 8 and at most 64 tokens, K <= 1024, N <= 1024, at most 8 Ki
  *       elements of A per CTA of a cluster of up to four; never while a configuration is forced or with SmoothQuant
  *       factors)
  *    0  never

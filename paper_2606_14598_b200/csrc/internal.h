@@ -94,7 +94,8 @@ cudaError_t launch_gemm_simt(const GemmArgs& a, cudaStream_t st);
 // ---- small_fused.cu : quantizer, GEMM and epilogue in one kernel, for problems of at most 128 tokens and K <= 1024
 constexpr int kSkinnyM = 8;           // at or below this many tokens the weight-streaming path runs
 constexpr int64_t kSmallFusedMaxCtas = 32;                 // 32-channel CTAs the one-kernel path is chosen for (N <= 1024)
-constexpr int64_t kSmallFusedMaxElemsPerCta = 16 << 10;    // elements of A one of its CTAs may have to quantize
+constexpr int64_t kSmallFusedMaxTokens = 64;               // tokens up to which it is chosen
+constexpr int64_t kSmallFusedMaxElemsPerCta = 8 << 10;     // elements of A one of its CTAs may have to quantize
 bool small_fused_eligible(int64_t M, int64_t N, int64_t K);     // what the kernel can run
 bool small_fused_preferred(int64_t M, int64_t N, int64_t K);    // where it is chosen when nothing is forced
 // Writes the codes and scales to qa_out / s_tok_out as the two-kernel path does, the output to g.out.

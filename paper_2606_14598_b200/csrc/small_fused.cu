@@ -324,12 +324,12 @@ bool small_fused_eligible(int64_t M, int64_t N, int64_t K) {
 }
 
 // Where it is the faster path (GPU time per call inside a CUDA graph of 50 calls, against the two-kernel path): more
-// than a handful of tokens (fewer go to the weight-streaming kernel, which is as fast there), at most 32 CTAs, and
-// at most 16 Ki elements of A to quantize per CTA (every cluster repeats the quantizer's work; M = 128:
-// K = N = 256 5.4 against 6.2 us, K = N = 512 6.5 against 7.1 us, K = N = 1024 9.4 against 8.5 us; M = 16,
-// K = 512, N = 1024 4.3 against 6.8 us).
+// than a handful of tokens (fewer go to the weight-streaming kernel, which is as fast there) and at most 64, at most
+// 32 CTAs, and at most 8 Ki elements of A to quantize per CTA (every cluster repeats the quantizer's work).
+// One kernel / two kernels: M = 16, K = 512, N = 1024 4.5 / 5.3 us; (32, 256, 256) 3.9 / 4.7; (64, 512, 512) 5.1 / 5.5;
+// (32, 1024, 1024) 6.1 / 6.6; but (64, 1024, 1024) 7.1 / 6.8, (128, 256, 256) 5.5 / 5.2, (128, 1024, 1024) 9.4 / 6.9.
 bool small_fused_preferred(int64_t M, int64_t N, int64_t K) {
-    if (!small_fused_eligible(M, N, K) || M <= kSkinnyM) return false;
+    if (!small_fused_eligible(M, N, K) || M <= kSkinnyM || M > kSmallFusedMaxTokens) return false;
     const int64_t ctas = (N + SF_BN - 1) / SF_BN;
     const int64_t cs = ctas >= 4 ? 4 : ctas >= 2 ? 2 : 1;
     return ctas <= kSmallFusedMaxCtas && M * K <= kSmallFusedMaxElemsPerCta * cs;

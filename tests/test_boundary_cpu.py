@@ -90,21 +90,23 @@ def test_plan_of_the_benchmark_shapes():
 
 
 def test_one_kernel_path_is_chosen_for_one_tile_problems_only():
-    """Host logic of the default mode: c1 and its like take the one-kernel path; larger or skinnier problems, forced
-    configurations and pre-quantized activations do not."""
+    """Host logic of the default mode: problems of a few dozen tokens and a small A take the one-kernel path; larger
+    or skinnier problems, forced configurations and pre-quantized activations do not."""
     ws_big = 1 << 30
     name = lambda M, N, K, a=w8.ACT_BF16: w8.int8_linear_plan(M, N, K, a, ws_big)["name"]
-    assert "one kernel" in name(128, 256, 256)          # c1
+    assert "one kernel" in name(64, 512, 512)
     assert "one kernel" in name(16, 1024, 512)
-    assert "one kernel" not in name(128, 256, 256, w8.ACT_INT8)
-    assert "one kernel" not in name(128, 1024, 1024)    # 32 Ki elements per CTA of a cluster of four
-    assert "one kernel" not in name(129, 256, 256)
+    assert "one kernel" in name(16, 64, 1024)           # N = 64: a cluster of two shares 16 Ki elements
+    assert "one kernel" not in name(32, 64, 1024)       # ... but not 32 Ki
+    assert "one kernel" not in name(64, 512, 512, w8.ACT_INT8)
+    assert "one kernel" not in name(64, 1024, 1024)     # 16 Ki elements per CTA of a cluster of four
+    assert "one kernel" not in name(128, 256, 256)      # c1: more than 64 tokens
     assert "one kernel" not in name(64, 2048, 256)      # N > 1024
     assert "one kernel" not in name(8, 256, 256)        # skinny: the weight-streaming kernel
     assert "one kernel" not in name(2816, 3072, 3072)
     w8.force_config(0)
     try:
-        assert "one kernel" not in name(128, 256, 256)
+        assert "one kernel" not in name(64, 512, 512)
     finally:
         w8.force_config(-1)
 
