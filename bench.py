@@ -61,16 +61,19 @@ import pynvml as nv
 nv.nvmlInit()
 h = nv.nvmlDeviceGetHandleByIndex(int(idx)) if idx.isdigit() else nv.nvmlDeviceGetHandleByUUID(idx)
 print(json.dumps({"max_mhz": float(nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM))}), flush=True)
+pw, mask, n = None, 0, 0
 while True:
     t = time.time()
     try:
         mhz = float(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
-        pw = nv.nvmlDeviceGetPowerUsage(h) / 1000.0
-        try:
-            mask = nv.nvmlDeviceGetCurrentClocksEventReasons(h)
-        except Exception:
-            mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(h)
-        sys.stdout.write(json.dumps({"t": t, "mhz": mhz, "w": pw, "mask": int(mask)}) + "\n")
+        if n % 4 == 0:      # the clock every round; power and clock-event reasons (slower queries) every fourth
+            pw = nv.nvmlDeviceGetPowerUsage(h) / 1000.0
+            try:
+                mask = nv.nvmlDeviceGetCurrentClocksEventReasons(h)
+            except Exception:
+                mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+        n += 1
+        sys.stdout.write(json.dumps({"t": t, "mhz": mhz, "w": pw, "mask": int(mask), "dt": time.time() - t}) + "\n")
         sys.stdout.flush()
     except Exception:
         pass
@@ -87,9 +90,9 @@ class ClockSampler:
                0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting", 0x100: "display_clock_setting",
                0x10: "sync_boost"}
 
-    def __init__(self, index: int, period_s: float = 0.002):
+    def __init__(self, index: int, period_s: float = 0.001):
         import subprocess
-        self.samples, self.power, self.reasons = [], [], set()
+        self.samples, self.power, self.reasons, self.times = [], [], set(), []
         self.max_mhz, self.t0, self.t1, self.proc, self.out = None, None, None, None, None
         visible = os.environ.get("CUDA_VISIBLE_DEVICES")
         tok = str(index)
@@ -152,6 +155,7 @@ class ClockSampler:
                 continue
             if "t" in d and self.t0 <= d["t"] <= self.t1:
                 self.samples.append(d["mhz"])
+                self.times.append(d["t"])
                 if d["w"] is not None:
                     self.power.append(d["w"])
                 for bit, name in self.REASONS.items():
@@ -163,6 +167,7 @@ class ClockSampler:
             return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["not sampled"], "samples": 0}
         return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
                 "reasons": sorted(self.reasons), "samples": len(self.samples),
+                "sample_period_ms": (self.times[-1] - self.times[0]) / (len(self.times) - 1) * 1e3 if len(self.times) > 1 else None,
                 "power_w_max": max(self.power) if self.power else None}
 
 
@@ -548,6 +553,20 @@ def main():
 
             tg = batch_time(gemm_only)
             stamp = w8.gemm_clock_stamps(ws8) if M > 8 else None
+            # the same launches on operands that do not toggle (all codes 1): what the kernel does when the data costs
+            # no power, i.e. how much of the time above is the clock the chip allows on real operands
+            const_ops = None
+            if not args.no_extras and M > 16:
+                L0 = rot[0]
+                ones_a = torch.ones((M, K), dtype=torch.int8, device=dev)
+                ones_w = torch.ones((N, K), dtype=torch.int8, device=dev)
+                c_args = (ones_a.data_ptr(), 1, K, views[0][1].data_ptr(), ones_w.data_ptr(), L0["s_ch"].data_ptr(),
+                          None if L0["bias"] is None else L0["bias"].data_ptr(), L0["out"].data_ptr(), N, M, N, K,
+                          ws8.data_ptr(), ws8.numel(), stream)
+                tc_ = batch_time(lambda: raw.int8_linear_fused(*c_args))
+                cst = w8.gemm_clock_stamps(ws8)
+                const_ops = {"us": tc_ * 1e6, "tops": spec.ops / tc_ / 1e12, "gemm_sm_mhz": cst[0] if cst else None}
+                del ones_a, ones_w
             tgh = batch_time(gemm_hot)
             tq = batch_time(quant_only)
             tq1 = batch_time(quant_one_pass)
@@ -562,6 +581,7 @@ def main():
                               "gemm_sm_mhz": stamp[0] if stamp else None,
                               "gemm_first_cta_us": stamp[1] * 1e6 if stamp else None,
                               "gemm_epilogue_hot_l2_us": tgh * 1e6, "gemm_epilogue_hot_l2_tops": spec.ops / tgh / 1e12,
+                              "gemm_epilogue_constant_operands": const_ops,
                               "quantizer_us": tq * 1e6, "quantizer_gbs": model.quantizer_bytes(M, K) / tq / 1e9,
                               "quantizer_given_absmax_us": tq1 * 1e6,
                               "quantizer_given_absmax_gbs": (model.quantizer_bytes(M, K) + 4 * M) / tq1 / 1e9})
